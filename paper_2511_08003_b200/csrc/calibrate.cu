@@ -1,0 +1,197 @@
+// Stage two (a): self-calibrated degradation test (Section 3.2.3, Eq. 7) per visual token,
+// followed by the compaction of the keep flags into ascending kept positions.
+//
+// Kernels:
+//   calibrate_cos_kernel  one warp per packed position: cos(hidden row, visual row), keep flag;
+//                         each CTA also writes how many of its positions survive
+//   write_kept_kernel     same chunks: chunk base = sum of earlier chunk counts, local scan,
+//                         ascending kept positions, per-sequence offsets, capacity check
+//   mean_cos_kernel       (optional) fixed-order mean of the cosines of each sequence
+#include "common.cuh"
+
+namespace sharpv {
+namespace {
+
+constexpr int kChunk = 256;             // packed positions per CTA (8 warps x 32 positions)
+
+__host__ __device__ inline size_t ws_flags_bytes(int64_t T) { return ((size_t)T + 255) / 256 * 256; }
+__host__ __device__ inline int64_t num_chunks(int64_t T) { return (T + kChunk - 1) / kChunk; }
+
+template <int DT>
+__global__ void __launch_bounds__(256)
+calibrate_cos_kernel(const char* __restrict__ hidden, int64_t hidden_row_bytes,
+                     const char* __restrict__ visual, int64_t visual_row_bytes, int nvec,
+                     int num_seqs, const int32_t* __restrict__ seq_offsets,
+                     const int32_t* __restrict__ vis_begin, const int32_t* __restrict__ vis_count,
+                     const int32_t* __restrict__ vis_offsets, int64_t T, int64_t total_visual, float M,
+                     float* __restrict__ out_cos, uint8_t* __restrict__ flags,
+                     int32_t* __restrict__ chunk_counts) {
+    using E = Elem<DT>;
+    constexpr int P = E::kPerVec;
+    __shared__ int warp_kept[8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t chunk_base = (int64_t)blockIdx.x * kChunk;
+    int kept_here = 0;
+    for (int q = 0; q < kChunk / 8; ++q) {
+        const int64_t p = chunk_base + warp * (kChunk / 8) + q;
+        if (p >= T) break;
+        const int b = upper_segment(seq_offsets, num_seqs, (int)p);
+        const int64_t local = p - __ldg(seq_offsets + b) - __ldg(vis_begin + b);
+        int keep = 1;
+        if (local >= 0 && local < __ldg(vis_count + b)) {
+            const int64_t vrow = (int64_t)__ldg(vis_offsets + b) + local;
+            if (vrow < total_visual) {
+                const char* ph = hidden + p * hidden_row_bytes;
+                const char* pv = visual + vrow * visual_row_bytes;
+                float shh = 0.f, svv = 0.f, shv = 0.f;
+                for (int v = lane; v < nvec; v += 32) {
+                    float h[P], x[P];
+                    E::widen(ld_stream(ph + (int64_t)v * 16), h);
+                    E::widen(ld_stream(pv + (int64_t)v * 16), x);
+#pragma unroll
+                    for (int j = 0; j < P; ++j) {
+                        shh = fmaf(h[j], h[j], shh);
+                        svv = fmaf(x[j], x[j], svv);
+                        shv = fmaf(h[j], x[j], shv);
+                    }
+                }
+                shh = warp_sum(shh); svv = warp_sum(svv); shv = warp_sum(shv);
+                const float nh = fmaxf(sqrtf(shh), kNormEps), nv = fmaxf(sqrtf(svv), kNormEps);
+                const float c = shv / (nh * nv);
+                keep = c < M ? 0 : 1;                       // Eq. 7: discard iff cos < M
+                if (lane == 0) out_cos[vrow] = c;
+            }
+        }
+        if (lane == 0) flags[p] = (uint8_t)keep;
+        kept_here += keep;
+    }
+    if (lane == 0) warp_kept[warp] = kept_here;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int tot = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) tot += warp_kept[i];
+        chunk_counts[blockIdx.x] = tot;
+    }
+}
+
+__global__ void __launch_bounds__(kChunk)
+write_kept_kernel(const uint8_t* __restrict__ flags, const int32_t* __restrict__ chunk_counts,
+                  int64_t T, int num_seqs, const int32_t* __restrict__ seq_offsets, int64_t capacity,
+                  int32_t* __restrict__ out_kept_pos, int32_t* __restrict__ out_kept_seq_offsets,
+                  int32_t* status_word) {
+    __shared__ int sm[kChunk / 32 + 1];
+    __shared__ int s_base;
+    const int c = blockIdx.x;
+    // kept positions before this chunk: fixed-order sum of the earlier chunk counts
+    int part = 0;
+    for (int i = threadIdx.x; i < c; i += kChunk) part += chunk_counts[i];
+    int total_before;
+    block_exclusive_scan<kChunk>(part, sm, total_before);
+    if (threadIdx.x == 0) s_base = total_before;
+    __syncthreads();
+    const int base = s_base;
+
+    const int64_t p = (int64_t)c * kChunk + threadIdx.x;
+    const int keep = p < T ? flags[p] : 0;
+    int chunk_total;
+    const int rank = block_exclusive_scan<kChunk>(keep, sm, chunk_total);
+    const int64_t j = (int64_t)base + rank;
+    if (keep && j < capacity) out_kept_pos[j] = (int32_t)p;
+
+    // sequences that start at this position (several when some are empty)
+    if (p < T) {
+        int b = upper_segment(seq_offsets, num_seqs, (int)p);
+        while (b >= 0 && __ldg(seq_offsets + b) == (int)p) {
+            out_kept_seq_offsets[b] = (int32_t)j;
+            --b;
+        }
+    }
+    if (c == gridDim.x - 1 && threadIdx.x == 0) {
+        const int64_t total = (int64_t)base + chunk_total;
+        // trailing empty sequences and the end marker
+        for (int b = num_seqs; b >= 0 && __ldg(seq_offsets + b) >= T; --b) out_kept_seq_offsets[b] = (int32_t)total;
+        if (total > capacity) report(status_word, SHARPV_ERR_CAPACITY);
+    }
+}
+
+__global__ void __launch_bounds__(256)
+mean_cos_kernel(const float* __restrict__ cosv, const int32_t* __restrict__ vis_count,
+                const int32_t* __restrict__ vis_offsets, int64_t total_visual, float* __restrict__ out_mean) {
+    __shared__ float part[8];
+    const int b = blockIdx.x;
+    const int n = vis_count[b];
+    const int64_t o = vis_offsets[b];
+    float s = 0.f;
+    for (int i = threadIdx.x; i < n; i += 256)
+        if (o + i < total_visual) s += cosv[o + i];
+    s = warp_sum(s);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) tot += part[i];
+        out_mean[b] = n > 0 ? tot / (float)n : 0.f;
+    }
+}
+
+}  // namespace
+}  // namespace sharpv
+
+using namespace sharpv;
+
+extern "C" size_t sharpv_kv_calibrate_prune_workspace_bytes(int64_t total_seq_tokens, int32_t num_seqs) {
+    (void)num_seqs;
+    if (total_seq_tokens <= 0) return 256;
+    return ws_flags_bytes(total_seq_tokens) + align_up((size_t)num_chunks(total_seq_tokens) * 4, 256);
+}
+
+extern "C" sharpv_status sharpv_kv_calibrate_prune(
+    const void* hidden, int64_t ld_hidden, const void* visual, int64_t ld_visual, sharpv_dtype dtype,
+    int32_t d, int32_t num_seqs, const int32_t* seq_offsets, const int32_t* vis_begin,
+    const int32_t* vis_count, const int32_t* vis_offsets, int64_t total_seq_tokens, int64_t total_visual,
+    float M, float* out_cos, float* out_mean_cos, int32_t* out_kept_pos, int32_t* out_kept_seq_offsets,
+    int64_t capacity, void* workspace, size_t workspace_bytes, int32_t* status_word, void* cuda_stream) {
+    if (!dtype_ok(dtype)) return SHARPV_ERR_UNSUPPORTED;
+    if (num_seqs < 1 || d < 1 || total_seq_tokens < 0 || total_visual < 0 || capacity < 0 || ld_hidden < d ||
+        ld_visual < d)
+        return SHARPV_ERR_INVALID_ARG;
+    if (!seq_offsets || !vis_begin || !vis_count || !vis_offsets || !out_kept_seq_offsets)
+        return SHARPV_ERR_INVALID_ARG;
+    if (total_seq_tokens >= (int64_t)1 << 31 || total_visual >= (int64_t)1 << 31) return SHARPV_ERR_UNSUPPORTED;
+    const int eb = elem_bytes(dtype);
+    if (((int64_t)d * eb) % 16 || (ld_hidden * eb) % 16 || (ld_visual * eb) % 16) return SHARPV_ERR_UNSUPPORTED;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (total_seq_tokens == 0) {
+        if (cudaMemsetAsync(out_kept_seq_offsets, 0, sizeof(int32_t) * (size_t)(num_seqs + 1), stream) != cudaSuccess)
+            return SHARPV_ERR_CUDA;
+        if (out_mean_cos &&
+            cudaMemsetAsync(out_mean_cos, 0, sizeof(float) * (size_t)num_seqs, stream) != cudaSuccess)
+            return SHARPV_ERR_CUDA;
+        return SHARPV_OK;
+    }
+    if (!hidden || !workspace || (capacity > 0 && !out_kept_pos)) return SHARPV_ERR_INVALID_ARG;
+    if (total_visual > 0 && (!visual || !out_cos)) return SHARPV_ERR_INVALID_ARG;
+    if (!aligned16(hidden) || !aligned16(visual) || !aligned16(workspace)) return SHARPV_ERR_UNSUPPORTED;
+    if (workspace_bytes < sharpv_kv_calibrate_prune_workspace_bytes(total_seq_tokens, num_seqs))
+        return SHARPV_ERR_WORKSPACE;
+
+    uint8_t* flags = (uint8_t*)workspace;
+    int32_t* chunk_counts = (int32_t*)((char*)workspace + ws_flags_bytes(total_seq_tokens));
+    const unsigned chunks = (unsigned)num_chunks(total_seq_tokens);
+    const int nvec = d * eb / 16;
+    if (dtype == SHARPV_F32)
+        calibrate_cos_kernel<SHARPV_F32><<<chunks, 256, 0, stream>>>(
+            (const char*)hidden, ld_hidden * eb, (const char*)visual, ld_visual * eb, nvec, num_seqs, seq_offsets,
+            vis_begin, vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, flags, chunk_counts);
+    else
+        calibrate_cos_kernel<SHARPV_BF16><<<chunks, 256, 0, stream>>>(
+            (const char*)hidden, ld_hidden * eb, (const char*)visual, ld_visual * eb, nvec, num_seqs, seq_offsets,
+            vis_begin, vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, flags, chunk_counts);
+    write_kept_kernel<<<chunks, kChunk, 0, stream>>>(flags, chunk_counts, total_seq_tokens, num_seqs, seq_offsets,
+                                                    capacity, out_kept_pos, out_kept_seq_offsets, status_word);
+    if (out_mean_cos)
+        mean_cos_kernel<<<num_seqs, 256, 0, stream>>>(out_cos, vis_count, vis_offsets, total_visual, out_mean_cos);
+    return launch_status();
+}

@@ -1,0 +1,131 @@
+// Shared device helpers of the SharpV CUDA library: 128-bit loads, exact widening of
+// bf16 / fp32 storage to fp32, warp and block reductions, argument checks.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sharpv.h"
+
+namespace sharpv {
+
+constexpr int kWarp = 32;
+constexpr float kNormEps = 1e-12f;      // v^ = v / max(||v||, kNormEps)
+
+// ---------------------------------------------------------------------------------------
+// host-side argument checks
+// ---------------------------------------------------------------------------------------
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int elem_bytes(sharpv_dtype dt) { return dt == SHARPV_F32 ? 4 : 2; }
+inline bool dtype_ok(sharpv_dtype dt) { return dt == SHARPV_F32 || dt == SHARPV_BF16; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline sharpv_status launch_status() {
+    return cudaGetLastError() == cudaSuccess ? SHARPV_OK : SHARPV_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------
+// 16-byte vectors of the storage type and their exact fp32 widening
+// ---------------------------------------------------------------------------------------
+template <int DT> struct Elem;
+
+template <> struct Elem<SHARPV_F32> {
+    static constexpr int kPerVec = 4;
+    static constexpr int kBytes = 4;
+    __device__ __forceinline__ static void widen(const uint4& v, float (&x)[4]) {
+        x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y);
+        x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+    }
+};
+
+template <> struct Elem<SHARPV_BF16> {
+    static constexpr int kPerVec = 8;
+    static constexpr int kBytes = 2;
+    // a bf16 is the upper half of an fp32: element 2j is the low half-word, 2j+1 the high one
+    __device__ __forceinline__ static void widen(const uint4& v, float (&x)[8]) {
+        x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xffff0000u);
+        x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xffff0000u);
+        x[4] = __uint_as_float(v.z << 16); x[5] = __uint_as_float(v.z & 0xffff0000u);
+        x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xffff0000u);
+    }
+};
+
+// streaming 128-bit load: read-only path, do not keep the line in L1
+__device__ __forceinline__ uint4 ld_stream(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// 128-bit load that may stay in L1/L2 (small tables, frame means)
+__device__ __forceinline__ uint4 ld_cached(const void* p) {
+    return __ldg(reinterpret_cast<const uint4*>(p));
+}
+
+__device__ __forceinline__ void st_stream(void* p, const uint4& v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// ---------------------------------------------------------------------------------------
+// reductions (fixed order: results do not depend on scheduling)
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ int warp_sum_int(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Exclusive scan of one int per thread over a block of NT threads (NT a multiple of 32,
+// at most 1024).  `total` receives the block sum.  `smem` holds NT/32 + 1 ints.
+template <int NT>
+__device__ __forceinline__ int block_exclusive_scan(int v, int* smem, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    if (lane == 31) smem[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        int w = lane < NT / 32 ? smem[lane] : 0;
+        int winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int n = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += n;
+        }
+        if (lane < NT / 32) smem[lane] = winc - w;      // exclusive warp offsets
+        if (lane == 31) smem[NT / 32] = winc;           // block total
+    }
+    __syncthreads();
+    int res = smem[warp] + inc - v;
+    total = smem[NT / 32];
+    __syncthreads();                                     // smem may be reused by the caller
+    return res;
+}
+
+// largest b with offsets[b] <= x, for an ascending table offsets[0..n] (offsets[0] <= x < offsets[n])
+__device__ __forceinline__ int upper_segment(const int32_t* __restrict__ offsets, int n, int x) {
+    int lo = 0, hi = n;          // answer in [lo, hi)
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (__ldg(offsets + mid) <= x) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ void report(int32_t* status_word, int code) {
+    if (status_word) atomicMax(status_word, code);
+}
+
+}  // namespace sharpv

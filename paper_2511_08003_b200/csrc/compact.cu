@@ -1,0 +1,111 @@
+// Stage two (b): K/V compaction (Section 3.2.3).  For every (layer, K|V, head) plane the rows
+// of the kept positions are copied, in order, to a dense prefix of the destination plane.
+// One index list serves all planes.
+#include "common.cuh"
+
+namespace sharpv {
+namespace {
+
+constexpr int kTileRows = 64;           // destination rows per CTA
+constexpr int kCompactThreads = 256;
+
+struct PlaneGeom {
+    int64_t src_layer, src_kv, src_head, src_token;     // bytes
+    int64_t dst_layer, dst_kv, dst_head, dst_token;     // bytes
+    int num_kv_heads, layer_begin, row_vecs;            // row_vecs = 16-byte vectors per row
+};
+
+__global__ void __launch_bounds__(kCompactThreads)
+kv_compact_kernel(const char* __restrict__ src, char* __restrict__ dst, PlaneGeom g,
+                  const int32_t* __restrict__ kept_pos, const int32_t* __restrict__ n_kept_ptr,
+                  int64_t capacity, int32_t* status_word) {
+    const int64_t n_all = __ldg(n_kept_ptr);
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && n_all > capacity)
+        report(status_word, SHARPV_ERR_CAPACITY);
+    const int64_t n = min(n_all, capacity);
+    const int64_t row0 = (int64_t)blockIdx.x * kTileRows;
+    if (row0 >= n) return;
+    const int plane = blockIdx.y;
+    const int l = g.layer_begin + plane / (2 * g.num_kv_heads);
+    const int kv = (plane / g.num_kv_heads) & 1;
+    const int h = plane % g.num_kv_heads;
+    const char* s = src + l * g.src_layer + kv * g.src_kv + h * g.src_head;
+    char* o = dst + l * g.dst_layer + kv * g.dst_kv + h * g.dst_head;
+
+    const int rows = (int)min((int64_t)kTileRows, n - row0);
+    const int total = rows * g.row_vecs;
+    for (int q0 = threadIdx.x; q0 < total; q0 += kCompactThreads * 4) {
+        uint4 r[4];
+        int64_t off[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int q = q0 + u * kCompactThreads;
+            if (q < total) {
+                const int rr = q / g.row_vecs, vv = q - rr * g.row_vecs;
+                const int64_t j = row0 + rr;
+                r[u] = ld_stream(s + (int64_t)__ldg(kept_pos + j) * g.src_token + (int64_t)vv * 16);
+                off[u] = j * g.dst_token + (int64_t)vv * 16;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int q = q0 + u * kCompactThreads;
+            if (q < total) st_stream(o + off[u], r[u]);
+        }
+    }
+}
+
+bool layout_ok(const sharpv_kv_layout* L) {
+    return L && L->num_layers >= 1 && L->num_kv_heads >= 1 && L->head_dim >= 1 && dtype_ok(L->dtype) &&
+           L->stride_layer >= 0 && L->stride_kv >= 0 && L->stride_head >= 0 && L->stride_token >= L->head_dim;
+}
+
+bool layout_aligned(const sharpv_kv_layout* L) {
+    const int64_t eb = elem_bytes(L->dtype);
+    return (L->head_dim * eb) % 16 == 0 && (L->stride_layer * eb) % 16 == 0 && (L->stride_kv * eb) % 16 == 0 &&
+           (L->stride_head * eb) % 16 == 0 && (L->stride_token * eb) % 16 == 0;
+}
+
+}  // namespace
+}  // namespace sharpv
+
+using namespace sharpv;
+
+extern "C" sharpv_status sharpv_kv_compact(
+    const void* kv_src, const sharpv_kv_layout* src_layout, void* kv_dst, const sharpv_kv_layout* dst_layout,
+    int32_t layer_begin, int32_t layer_end, const int32_t* kept_pos, const int32_t* kept_seq_offsets,
+    int32_t num_seqs, int64_t capacity, int32_t* status_word, void* cuda_stream) {
+    if (!layout_ok(src_layout) || !layout_ok(dst_layout)) {
+        if (src_layout && dst_layout && (!dtype_ok(src_layout->dtype) || !dtype_ok(dst_layout->dtype)))
+            return SHARPV_ERR_UNSUPPORTED;
+        return SHARPV_ERR_INVALID_ARG;
+    }
+    if (src_layout->dtype != dst_layout->dtype || src_layout->head_dim != dst_layout->head_dim ||
+        src_layout->num_kv_heads != dst_layout->num_kv_heads || src_layout->num_layers != dst_layout->num_layers)
+        return SHARPV_ERR_INVALID_ARG;
+    if (layer_begin < 0 || layer_end > src_layout->num_layers || layer_begin > layer_end || num_seqs < 1 ||
+        capacity < 0)
+        return SHARPV_ERR_INVALID_ARG;
+    if (!kv_src || !kv_dst || !kept_seq_offsets || kv_src == kv_dst) return SHARPV_ERR_INVALID_ARG;
+    if (capacity > 0 && !kept_pos) return SHARPV_ERR_INVALID_ARG;
+    if (!layout_aligned(src_layout) || !layout_aligned(dst_layout) || !aligned16(kv_src) || !aligned16(kv_dst))
+        return SHARPV_ERR_UNSUPPORTED;
+    if (capacity >= (int64_t)1 << 31) return SHARPV_ERR_UNSUPPORTED;
+    const int planes = (layer_end - layer_begin) * 2 * src_layout->num_kv_heads;
+    if (planes == 0 || capacity == 0) return SHARPV_OK;
+    if (planes > 65535) return SHARPV_ERR_UNSUPPORTED;
+
+    const int64_t eb = elem_bytes(src_layout->dtype);
+    PlaneGeom g;
+    g.src_layer = src_layout->stride_layer * eb; g.src_kv = src_layout->stride_kv * eb;
+    g.src_head = src_layout->stride_head * eb;   g.src_token = src_layout->stride_token * eb;
+    g.dst_layer = dst_layout->stride_layer * eb; g.dst_kv = dst_layout->stride_kv * eb;
+    g.dst_head = dst_layout->stride_head * eb;   g.dst_token = dst_layout->stride_token * eb;
+    g.num_kv_heads = src_layout->num_kv_heads;
+    g.layer_begin = layer_begin;
+    g.row_vecs = (int)(src_layout->head_dim * eb / 16);
+    dim3 grid((unsigned)((capacity + kTileRows - 1) / kTileRows), (unsigned)planes);
+    kv_compact_kernel<<<grid, kCompactThreads, 0, (cudaStream_t)cuda_stream>>>(
+        (const char*)kv_src, (char*)kv_dst, g, kept_pos, kept_seq_offsets + num_seqs, capacity, status_word);
+    return launch_status();
+}

@@ -1,0 +1,263 @@
+// Stage one (b): per-frame top-k of the importance scores with a stable tie-break, the
+// exclusive scan of the budgets, and the gather of the kept token rows
+// (Section 3.1, first paragraph; Section 3.1.3, last paragraph).
+//
+// Kernels:
+//   count_above_kernel   (threshold variant only) per-frame count of I > K
+//   scan_budgets_kernel  one CTA: exclusive scan of the clamped budgets -> kept_offsets
+//   select_frame_kernel  one CTA per frame: radix select of the k-th largest key in shared
+//                        memory, then an index-ordered scan that writes ascending indices
+//   gather_rows_kernel   one warp per kept row, 128-bit copies
+#include "common.cuh"
+
+namespace sharpv {
+namespace {
+
+constexpr int kSelectThreads = 256;
+constexpr int kMaxTokensPerFrame = 8192;
+
+// Monotone map fp32 -> uint32: larger score, larger key.  Adding +0 turns -0 into +0.
+__device__ __forceinline__ uint32_t order_key(float x) {
+    const uint32_t b = __float_as_uint(x + 0.0f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+__global__ void __launch_bounds__(kSelectThreads)
+count_above_kernel(const float* __restrict__ importance, float K, int f, int32_t* __restrict__ counts) {
+    __shared__ int part[kSelectThreads / 32];
+    const int t = blockIdx.x;
+    int c = 0;
+    for (int i = threadIdx.x; i < f; i += kSelectThreads) c += importance[(int64_t)t * f + i] > K;
+    c = warp_sum_int(c);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int tot = 0;
+        for (int i = 0; i < kSelectThreads / 32; ++i) tot += part[i];
+        counts[t] = tot;
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+scan_budgets_kernel(const int32_t* __restrict__ k, int F, int f, int64_t capacity,
+                    int32_t* __restrict__ kept_offsets, int32_t* __restrict__ num_kept,
+                    int32_t* status_word) {
+    __shared__ int sm[1024 / 32 + 1];
+    int carry = 0;
+    for (int base = 0; base < F; base += 1024) {
+        const int t = base + threadIdx.x;
+        int v = 0;
+        if (t < F) v = min(max(k[t], 0), f);
+        int total;
+        const int ex = block_exclusive_scan<1024>(v, sm, total);
+        if (t < F) kept_offsets[t] = carry + ex;
+        carry += total;
+    }
+    if (threadIdx.x == 0) {
+        kept_offsets[F] = carry;
+        if (num_kept) *num_kept = carry;
+        if ((int64_t)carry > capacity) report(status_word, SHARPV_ERR_CAPACITY);
+    }
+}
+
+// mode 0: top-k with budgets k[t];  mode 1: keep I > K
+__global__ void __launch_bounds__(kSelectThreads)
+select_frame_kernel(const float* __restrict__ importance, const int32_t* __restrict__ k,
+                    const int32_t* __restrict__ kept_offsets, int f, int64_t capacity, int mode, float K,
+                    int32_t* __restrict__ out_kept_index) {
+    extern __shared__ uint32_t keys[];                 // [f]
+    __shared__ int hist[256];
+    __shared__ int scan_sm[kSelectThreads / 32 + 1];
+    __shared__ int s_digit, s_remaining;
+
+    const int t = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t out_base = kept_offsets[t];
+    const float* imp = importance + (int64_t)t * f;
+
+    uint32_t kth = 0;
+    int remaining = 0;
+    bool keep_all = false;
+    if (mode == 0) {
+        const int kt = min(max(k[t], 0), f);
+        if (kt == 0) return;
+        keep_all = kt == f;
+        for (int i = tid; i < f; i += kSelectThreads) keys[i] = order_key(imp[i]);
+        __syncthreads();
+        if (!keep_all) {
+            // radix select, most significant byte first: after the four passes `prefix` is the
+            // k-th largest key and `remaining` says how many keys equal to it are still owed
+            uint32_t prefix = 0, mask = 0;
+            remaining = kt;
+            for (int shift = 24; shift >= 0; shift -= 8) {
+                for (int i = tid; i < 256; i += kSelectThreads) hist[i] = 0;
+                __syncthreads();
+                for (int i = tid; i < f; i += kSelectThreads) {
+                    const uint32_t key = keys[i];
+                    if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+                }
+                __syncthreads();
+                if (warp == 0) {
+                    const int top = 255 - lane * 8;    // lane 0 owns the 8 largest digits
+                    int c[8], sum = 0;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) { c[j] = hist[top - j]; sum += c[j]; }
+                    int inc = sum;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        int n = __shfl_up_sync(0xffffffffu, inc, o);
+                        if (lane >= o) inc += n;
+                    }
+                    int acc = inc - sum;               // candidates with a larger digit than my range
+                    if (acc < remaining && remaining <= inc) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            if (acc < remaining && remaining <= acc + c[j]) {
+                                s_digit = top - j;
+                                s_remaining = remaining - acc;
+                            }
+                            acc += c[j];
+                        }
+                    }
+                }
+                __syncthreads();
+                prefix |= (uint32_t)s_digit << shift;
+                mask |= 0xffu << shift;
+                remaining = s_remaining;
+            }
+            kth = prefix;
+        }
+    } else {
+        // threshold variant: key 1 for kept, 0 otherwise; "greater than 0" keeps them
+        for (int i = tid; i < f; i += kSelectThreads) keys[i] = imp[i] > K ? 1u : 0u;
+        __syncthreads();
+        kth = 0;
+        remaining = 0;
+    }
+
+    // index-ordered pass: keys above the k-th are kept; among keys equal to it the first
+    // `remaining` in index order are kept
+    int carry_eq = 0, carry_keep = 0;
+    for (int base = 0; base < f; base += kSelectThreads) {
+        const int i = base + tid;
+        const bool valid = i < f;
+        const uint32_t key = valid ? keys[i] : 0u;
+        bool keep;
+        if (keep_all) {
+            keep = valid;
+        } else {
+            const bool gt = valid && key > kth;
+            const int eq = (valid && key == kth && remaining > 0) ? 1 : 0;
+            int tot_eq;
+            const int eq_rank = carry_eq + block_exclusive_scan<kSelectThreads>(eq, scan_sm, tot_eq);
+            carry_eq += tot_eq;
+            keep = gt || (eq && eq_rank < remaining);
+        }
+        int tot_keep;
+        const int pos = carry_keep + block_exclusive_scan<kSelectThreads>(keep ? 1 : 0, scan_sm, tot_keep);
+        carry_keep += tot_keep;
+        if (keep) {
+            const int64_t j = out_base + pos;
+            if (j < capacity) out_kept_index[j] = t * f + i;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const char* __restrict__ src, int64_t src_row_bytes, int nvec,
+                   const int32_t* __restrict__ index, const int32_t* __restrict__ count_ptr,
+                   int64_t capacity, char* __restrict__ dst, int64_t dst_row_bytes) {
+    const int lane = threadIdx.x & 31;
+    const int64_t j = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int64_t n = min((int64_t)__ldg(count_ptr), capacity);
+    if (j >= n) return;
+    const char* s = src + (int64_t)__ldg(index + j) * src_row_bytes;
+    char* o = dst + j * dst_row_bytes;
+    int v = lane;
+    for (; v + 96 < nvec; v += 128) {
+        uint4 r0 = ld_stream(s + (int64_t)v * 16);
+        uint4 r1 = ld_stream(s + (int64_t)(v + 32) * 16);
+        uint4 r2 = ld_stream(s + (int64_t)(v + 64) * 16);
+        uint4 r3 = ld_stream(s + (int64_t)(v + 96) * 16);
+        st_stream(o + (int64_t)v * 16, r0);
+        st_stream(o + (int64_t)(v + 32) * 16, r1);
+        st_stream(o + (int64_t)(v + 64) * 16, r2);
+        st_stream(o + (int64_t)(v + 96) * 16, r3);
+    }
+    for (; v < nvec; v += 32) st_stream(o + (int64_t)v * 16, ld_stream(s + (int64_t)v * 16));
+}
+
+sharpv_status select_impl(int mode, const float* importance, const int32_t* k, float K, int32_t F, int32_t f,
+                          const void* tokens, sharpv_dtype dtype, int64_t ld_tokens, int32_t d,
+                          int32_t* out_kept_index, int32_t* out_kept_offsets, void* out_tokens,
+                          int64_t capacity, int32_t* out_num_kept, void* workspace, size_t workspace_bytes,
+                          int32_t* status_word, void* cuda_stream) {
+    if (F < 0 || f < 1 || capacity < 0) return SHARPV_ERR_INVALID_ARG;
+    if (!out_kept_offsets) return SHARPV_ERR_INVALID_ARG;
+    if (f > kMaxTokensPerFrame) return SHARPV_ERR_UNSUPPORTED;
+    if ((int64_t)F * f >= (int64_t)1 << 31) return SHARPV_ERR_UNSUPPORTED;
+    if (F > 0 && (!importance || (mode == 0 && !k))) return SHARPV_ERR_INVALID_ARG;
+    if (capacity > 0 && !out_kept_index) return SHARPV_ERR_INVALID_ARG;
+    int eb = 0;
+    if (out_tokens) {
+        if (!dtype_ok(dtype)) return SHARPV_ERR_UNSUPPORTED;
+        if (!tokens || d < 1 || ld_tokens < d) return SHARPV_ERR_INVALID_ARG;
+        eb = elem_bytes(dtype);
+        if (((int64_t)d * eb) % 16 || (ld_tokens * eb) % 16 || !aligned16(tokens) || !aligned16(out_tokens))
+            return SHARPV_ERR_UNSUPPORTED;
+    }
+    if (workspace_bytes < sharpv_select_tokens_workspace_bytes(F, f)) return SHARPV_ERR_WORKSPACE;
+    if (F > 0 && !workspace) return SHARPV_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+    const int32_t* budgets = k;
+    if (mode == 1 && F > 0) {
+        int32_t* counts = (int32_t*)workspace;
+        count_above_kernel<<<F, kSelectThreads, 0, stream>>>(importance, K, f, counts);
+        budgets = counts;
+    }
+    scan_budgets_kernel<<<1, 1024, 0, stream>>>(budgets, F, f, capacity, out_kept_offsets, out_num_kept,
+                                                status_word);
+    if (F > 0) {
+        select_frame_kernel<<<F, kSelectThreads, (size_t)f * 4, stream>>>(
+            importance, budgets, out_kept_offsets, f, capacity, mode, K, out_kept_index);
+        if (out_tokens && capacity > 0) {
+            const int64_t rows = capacity < (int64_t)F * f ? capacity : (int64_t)F * f;
+            const int nvec = d * eb / 16;
+            gather_rows_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, stream>>>(
+                (const char*)tokens, ld_tokens * eb, nvec, out_kept_index, out_kept_offsets + F, capacity,
+                (char*)out_tokens, (int64_t)d * eb);
+        }
+    }
+    return launch_status();
+}
+
+}  // namespace
+}  // namespace sharpv
+
+using namespace sharpv;
+
+extern "C" size_t sharpv_select_tokens_workspace_bytes(int32_t total_frames, int32_t f) {
+    (void)f;
+    return align_up((size_t)(total_frames > 0 ? total_frames : 1) * 4, 256);
+}
+
+extern "C" sharpv_status sharpv_select_tokens(
+    const float* importance, const int32_t* k, int32_t total_frames, int32_t f, const void* tokens,
+    sharpv_dtype dtype, int64_t ld_tokens, int32_t d, int32_t* out_kept_index, int32_t* out_kept_offsets,
+    void* out_tokens, int64_t capacity, int32_t* out_num_kept, void* workspace, size_t workspace_bytes,
+    int32_t* status_word, void* cuda_stream) {
+    return select_impl(0, importance, k, 0.f, total_frames, f, tokens, dtype, ld_tokens, d, out_kept_index,
+                       out_kept_offsets, out_tokens, capacity, out_num_kept, workspace, workspace_bytes,
+                       status_word, cuda_stream);
+}
+
+extern "C" sharpv_status sharpv_select_tokens_threshold(
+    const float* importance, float K, int32_t total_frames, int32_t f, const void* tokens,
+    sharpv_dtype dtype, int64_t ld_tokens, int32_t d, int32_t* out_kept_index, int32_t* out_kept_offsets,
+    void* out_tokens, int64_t capacity, int32_t* out_num_kept, void* workspace, size_t workspace_bytes,
+    int32_t* status_word, void* cuda_stream) {
+    return select_impl(1, importance, nullptr, K, total_frames, f, tokens, dtype, ld_tokens, d, out_kept_index,
+                       out_kept_offsets, out_tokens, capacity, out_num_kept, workspace, workspace_bytes,
+                       status_word, cuda_stream);
+}

@@ -1,0 +1,334 @@
+"""GPU parity: every C-ABI entry point against the CPU oracle, element by element, on the same
+seeded inputs.  Runs on a B200 (`-m gpu`)."""
+import functools
+
+import numpy as np
+import pytest
+import torch
+
+from helpers import (BOUNDARY_TOL, TIGHT_TOL, TOL, DeviceWorkload, check_budgets, check_kept_sets, rel_err,
+                     to_dev, to_host)
+from oracle import sharpv_oracle as orc
+from paper_2511_08003_b200 import binding as sv
+from paper_2511_08003_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+NT = 8  # oracle threads
+
+
+def _small_ragged():
+    vids = [W.make_video_spec(5, 0.9, cuts=[2]), W.make_video_spec(1, 0.5), W.make_video_spec(9, 0.75, cuts=[3, 4]),
+            W.make_video_spec(2, 0.99)]
+    return W.custom("small_ragged", 40, W.BF16, 14, 3584, 64, vids, 0.0, 3, 4, 128)
+
+
+def _odd_shapes():
+    # f = 37 (not a multiple of anything), d = 8 fp32 (one 32-byte row), head_dim 8
+    vids = [W.make_video_spec(7, 0.6, cuts=[5], duplicates=[2]), W.make_video_spec(3, 0.3)]
+    wl = W.custom("odd", 41, W.F32, 6, 8, 3, vids, 0.0, 2, 3, 8)
+    return wl
+
+
+CASES = {
+    "tiny": lambda: W.tiny(),
+    "onevision_small": lambda: W.onevision_7b(n_frames=8, num_layers=2),
+    "video7b_small": lambda: W.video_7b(n_frames=16, num_layers=2),
+    "small_ragged": _small_ragged,
+    "odd_shapes": _odd_shapes,
+    "pllava_like": lambda: W.custom("pllava", 42, W.BF16, 12, 4096, 20, [W.make_video_spec(4, 0.9)], 0.0, 2, 8, 128),
+    "onevision_7b": lambda: W.onevision_7b(),
+    "video_7b": lambda: W.video_7b(),
+}
+
+
+@functools.lru_cache(maxsize=None)
+def _case(name):
+    wl = CASES[name]()
+    W.fill_tokens(wl)
+    W.fill_hidden(wl)
+    if wl.kv_bytes() <= 1 << 30:
+        W.fill_kv(wl)
+    return wl, DeviceWorkload(wl, kv=True)
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_stage_one_scores_budgets_selection_gather(name):
+    wl, dw = _case(name)
+    F, f = wl.total_frames, wl.f
+    o = orc.score_frames(wl.tokens, wl.video_frame_offsets, f, w=1.0, nthreads=NT)
+    g = sv.sharpv_score_frames(dw.tokens, dw.video_frame_offsets, F, f, w=1.0, want_spatial=True,
+                               want_temporal=True)
+    torch.cuda.synchronize()
+    tol = TOL[wl.dtype]
+    for key in ("spatial", "temporal", "importance"):
+        e = rel_err(to_host(g[key]), o[key])
+        assert e <= tol, f"{key}: rel err {e}"
+        assert e <= TIGHT_TOL, f"{key}: rel err {e} (fp32-accumulation bound)"
+    assert rel_err(to_host(g["ratio"]), o["ratio"]) <= TIGHT_TOL
+    k_gpu = to_host(g["k"])
+    exempt_frames = check_budgets(k_gpu, o, f)
+    assert len(exempt_frames) <= max(1, F // 50)
+
+    # exact duplicates give exactly zero temporal importance and an empty budget
+    for v, off in zip(wl.videos, wl.video_frame_offsets[:-1]):
+        for t in np.nonzero(v.duplicate)[0]:
+            assert np.all(to_host(g["temporal"])[(off + t) * f:(off + t + 1) * f] == 0.0)
+            assert k_gpu[off + t] == 0
+
+    sel = sv.sharpv_select_tokens(g["importance"], g["k"], F, f, tokens=dw.tokens)
+    torch.cuda.synchronize()
+    n = int(sel["num_kept"].item())
+    assert n == int(k_gpu.sum())                                   # kept count = sum of budgets
+    idx = to_host(sel["kept_index"])[:n]
+    off = to_host(sel["kept_offsets"])
+    exempt = check_kept_sets(idx, off, o["importance"], k_gpu, f, orc.select_tokens)
+    assert exempt <= max(2, n // 1000)
+    # gathered rows are a bit copy of the rows the GPU selected
+    np.testing.assert_array_equal(to_host(sel["tokens"])[:n], orc.gather_rows(wl.tokens, idx))
+
+
+@pytest.mark.parametrize("name", ["tiny", "small_ragged", "odd_shapes"])
+@pytest.mark.parametrize("kind", [sv.DISSIM, sv.ONE_MINUS_COS])
+@pytest.mark.parametrize("round_mode,min_keep,w", [(sv.ROUND_FLOOR, 0, 1.0), (sv.ROUND_NEAREST, 3, 0.5),
+                                                   (sv.ROUND_CEIL, 0, 2.0)])
+def test_score_variants(name, kind, round_mode, min_keep, w):
+    wl, dw = _case(name)
+    F, f = wl.total_frames, wl.f
+    o = orc.score_frames(wl.tokens, wl.video_frame_offsets, f, w=w, round_mode=round_mode, min_keep=min_keep,
+                         dissim_kind=kind, nthreads=NT)
+    g = sv.sharpv_score_frames(dw.tokens, dw.video_frame_offsets, F, f, w=w, dissim_kind=kind,
+                               round_mode=round_mode, min_keep=min_keep)
+    torch.cuda.synchronize()
+    assert "spatial" not in g and "temporal" not in g
+    assert rel_err(to_host(g["importance"]), o["importance"]) <= TIGHT_TOL
+    assert rel_err(to_host(g["ratio"]), o["ratio"]) <= TIGHT_TOL
+    check_budgets(to_host(g["k"]), o, f)
+
+
+def test_select_alone_is_bit_exact_with_ties():
+    """Same fp32 scores and budgets on both sides: no tolerance, ties included."""
+    rng = np.random.default_rng(50)
+    for F, f in ((1, 1), (3, 7), (40, 196), (5, 1000), (2, 8192), (300, 169)):
+        imp = rng.standard_normal(F * f).astype(np.float32)
+        imp[rng.integers(0, F * f, F * f // 3)] = 0.25           # heavy ties
+        imp[rng.integers(0, F * f, 5)] = -0.0
+        imp[rng.integers(0, F * f, 5)] = 0.0
+        if F > 2:
+            imp[f:2 * f] = 1.0                                   # a frame of equal scores
+        k = rng.integers(0, f + 1, F).astype(np.int32)
+        k[0] = f if F > 1 else k[0]
+        k[-1] = 0 if F > 1 else k[-1]
+        idx_o, off_o = orc.select_tokens(imp, k, f)
+        g = sv.sharpv_select_tokens(torch.from_numpy(imp).cuda(), torch.from_numpy(k).cuda(), F, f, gather=False)
+        torch.cuda.synchronize()
+        n = int(g["num_kept"].item())
+        np.testing.assert_array_equal(to_host(g["kept_offsets"]), off_o)
+        np.testing.assert_array_equal(to_host(g["kept_index"])[:n], idx_o)
+        # budgets out of range are clamped to [0, f]
+        k2 = k.copy()
+        k2[0] = f + 5
+        k2[-1] = -3
+        g2 = sv.sharpv_select_tokens(torch.from_numpy(imp).cuda(), torch.from_numpy(k2).cuda(), F, f, gather=False)
+        idx_o2, off_o2 = orc.select_tokens(imp, k2, f)
+        np.testing.assert_array_equal(to_host(g2["kept_offsets"]), off_o2)
+        np.testing.assert_array_equal(to_host(g2["kept_index"])[:off_o2[-1]], idx_o2)
+
+
+def test_select_threshold_variant():
+    wl, dw = _case("tiny")
+    F, f = wl.total_frames, wl.f
+    g = sv.sharpv_score_frames(dw.tokens, dw.video_frame_offsets, F, f, dissim_kind=sv.ONE_MINUS_COS)
+    imp = to_host(g["importance"])
+    for K in (0.0, 0.1, float(np.median(imp)), 1.6, 10.0):
+        idx_o, off_o = orc.select_threshold(imp, K, F, f)
+        s = sv.sharpv_select_tokens_threshold(g["importance"], K, F, f, tokens=dw.tokens)
+        torch.cuda.synchronize()
+        n = int(s["num_kept"].item())
+        assert n == idx_o.size
+        np.testing.assert_array_equal(to_host(s["kept_offsets"]), off_o)
+        np.testing.assert_array_equal(to_host(s["kept_index"])[:n], idx_o)
+        np.testing.assert_array_equal(to_host(s["tokens"])[:n], wl.tokens[idx_o])
+
+
+@pytest.mark.parametrize("name", list(CASES))
+@pytest.mark.parametrize("M", [0.2, 0.788, 0.95])
+def test_stage_two_calibration_and_compaction(name, M):
+    wl, dw = _case(name)
+    T = wl.total_seq_tokens
+    o = orc.kv_calibrate_prune(wl.hidden, wl.tokens, wl.seq_offsets, wl.vis_begin, wl.vis_count, wl.vis_offsets,
+                               M, nthreads=NT)
+    g = sv.sharpv_kv_calibrate_prune(dw.hidden, dw.tokens, dw.seq_offsets, dw.vis_begin, dw.vis_count,
+                                     dw.vis_offsets, T, M=M, want_mean_cos=True)
+    torch.cuda.synchronize()
+    cos_g = to_host(g["cos"])[:wl.n_visual]
+    e = rel_err(cos_g, o["cos"])
+    assert e <= TIGHT_TOL, f"cos rel err {e}"
+    kso = to_host(g["kept_seq_offsets"])
+    n = int(kso[-1])
+    kept = to_host(g["kept_pos"])[:n]
+    assert np.all(np.diff(kept) > 0)
+    sym = np.setxor1d(kept, o["kept_pos"])
+    if sym.size:                                                   # only tokens at the threshold may differ
+        vis_row = np.full(T, -1)
+        for b in range(wl.num_videos):
+            s0 = wl.seq_offsets[b] + wl.vis_begin[b]
+            vis_row[s0:s0 + wl.vis_count[b]] = wl.vis_offsets[b] + np.arange(wl.vis_count[b])
+        assert np.all(vis_row[sym] >= 0)
+        assert np.all(np.abs(o["cos"][vis_row[sym]] - M) <= BOUNDARY_TOL)
+        assert sym.size <= max(2, wl.n_visual // 1000)
+    else:
+        np.testing.assert_array_equal(kso, o["kept_seq_offsets"])
+    # the flags the GPU used are consistent with its own cosines
+    for b in range(wl.num_videos):
+        seg = kept[kso[b]:kso[b + 1]]
+        assert np.all((seg >= wl.seq_offsets[b]) & (seg < wl.seq_offsets[b + 1]))
+    mean_o = [o["cos"][wl.vis_offsets[b]:wl.vis_offsets[b] + wl.vis_count[b]].mean() for b in range(wl.num_videos)]
+    assert rel_err(to_host(g["mean_cos"]), np.array(mean_o)) <= 1e-5
+
+    if wl.kv is None:
+        return
+    dst = torch.zeros_like(dw.kv)
+    sv.sharpv_kv_compact(dw.kv, dst, g["kept_pos"], g["kept_seq_offsets"], capacity=T)
+    torch.cuda.synchronize()
+    expect = orc.kv_compact(wl.kv, kept, nthreads=NT)             # for the GPU's own index set
+    np.testing.assert_array_equal(to_host(dst), expect)           # bit exact, rows beyond n untouched (zero)
+
+
+def test_kv_compact_layouts_and_layer_range():
+    wl, dw = _case("small_ragged")
+    T = wl.total_seq_tokens
+    rng = np.random.default_rng(51)
+    kept = np.sort(rng.choice(T, size=T // 3, replace=False)).astype(np.int32)
+    kept_d = torch.from_numpy(kept).cuda()
+    kso = torch.tensor([0, kept.size], dtype=torch.int32, device="cuda")
+    L, _, H, _, Dh = wl.kv_shape()
+    # token-major source [L,2,T,H,Dh] viewed as [L,2,H,T,Dh]; smaller destination capacity
+    src_tm = dw.kv.permute(0, 1, 3, 2, 4).contiguous()
+    cap = kept.size + 5
+    dst = torch.zeros((L, 2, H, cap, Dh), dtype=dw.kv.dtype, device="cuda")
+    sv.sharpv_kv_compact(src_tm.permute(0, 1, 3, 2, 4), dst, kept_d, kso, capacity=cap, layer_begin=1, layer_end=3)
+    torch.cuda.synchronize()
+    out = to_host(dst)
+    assert np.all(out[0] == 0)
+    np.testing.assert_array_equal(out[1:3, :, :, :kept.size], wl.kv[1:3][:, :, :, kept])
+    assert np.all(out[:, :, :, kept.size:] == 0)
+    # token-major destination
+    dst_tm = torch.zeros((L, 2, cap, H, Dh), dtype=dw.kv.dtype, device="cuda")
+    sv.sharpv_kv_compact(dw.kv, dst_tm.permute(0, 1, 3, 2, 4), kept_d, kso, capacity=cap)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(to_host(dst_tm)[:, :, :kept.size], wl.kv[:, :, :, kept].transpose(0, 1, 3, 2, 4))
+
+
+def test_capacity_overflow_is_reported_not_written():
+    wl, dw = _case("tiny")
+    F, f, T = wl.total_frames, wl.f, wl.total_seq_tokens
+    g = sv.sharpv_score_frames(dw.tokens, dw.video_frame_offsets, F, f)
+    full = sv.sharpv_select_tokens(g["importance"], g["k"], F, f, tokens=dw.tokens)
+    n = int(full["num_kept"].item())
+    cap = n - 7
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    guard = 12345
+    out = {"kept_index": torch.full((cap + 16,), guard, dtype=torch.int32, device="cuda"),
+           "tokens": torch.zeros((cap + 16, wl.d), dtype=dw.tokens.dtype, device="cuda")}
+    s = sv.sharpv_select_tokens(g["importance"], g["k"], F, f, tokens=dw.tokens, capacity=cap, out=out,
+                                status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == sv.Status.ERR_CAPACITY
+    assert int(s["num_kept"].item()) == n                          # true count still reported
+    np.testing.assert_array_equal(to_host(s["kept_index"])[:cap], to_host(full["kept_index"])[:cap])
+    assert np.all(to_host(s["kept_index"])[cap:] == guard)         # nothing written beyond capacity
+    assert np.all(to_host(s["tokens"])[cap:] == 0)
+    np.testing.assert_array_equal(to_host(s["tokens"])[:cap], to_host(full["tokens"])[:cap])
+
+    status.zero_()
+    c = sv.sharpv_kv_calibrate_prune(dw.hidden, dw.tokens, dw.seq_offsets, dw.vis_begin, dw.vis_count,
+                                     dw.vis_offsets, T, M=0.2, capacity=100,
+                                     out={"kept_pos": torch.full((132,), guard, dtype=torch.int32, device="cuda")},
+                                     status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == sv.Status.ERR_CAPACITY
+    assert int(c["kept_seq_offsets"][-1].item()) == T              # everything survives M = 0.2 here
+    np.testing.assert_array_equal(to_host(c["kept_pos"])[:100], np.arange(100))
+    assert np.all(to_host(c["kept_pos"])[100:] == guard)
+    status.zero_()
+    dst = torch.zeros_like(dw.kv)
+    sv.sharpv_kv_compact(dw.kv, dst, c["kept_pos"], c["kept_seq_offsets"], capacity=100, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == sv.Status.ERR_CAPACITY
+    np.testing.assert_array_equal(to_host(dst)[:, :, :, :100], wl.kv[:, :, :, :100])
+    assert np.all(to_host(dst)[:, :, :, 100:] == 0)
+
+
+def test_degenerate_inputs():
+    dev = "cuda"
+    # no frames at all
+    vfo = torch.zeros(2, dtype=torch.int32, device=dev)
+    tok = torch.zeros((4, 8), dtype=torch.float32, device=dev)
+    g = sv.sharpv_score_frames(tok, vfo, 0, 4)
+    assert g["importance"].numel() == 0
+    s = sv.sharpv_select_tokens(g["importance"], g["k"], 0, 4, gather=False)
+    torch.cuda.synchronize()
+    assert int(s["num_kept"].item()) == 0 and to_host(s["kept_offsets"]).tolist() == [0]
+    # one token per frame, zero vectors, a uniform frame (every token equals the mean)
+    f, d = 4, 16
+    x = np.zeros((3 * f, d), np.float32)
+    x[f:2 * f] = np.arange(1, d + 1, dtype=np.float32)             # uniform frame: S = 0 exactly in the oracle
+    x[2 * f:3 * f] = np.random.default_rng(52).standard_normal((f, d)).astype(np.float32)
+    x[2 * f + 1] = 0.0                                              # a zero token inside a normal frame
+    o = orc.score_frames(x, [0, 3], f)
+    g = sv.sharpv_score_frames(to_dev(x), torch.tensor([0, 3], dtype=torch.int32, device=dev), 3, f,
+                               want_spatial=True, want_temporal=True)
+    torch.cuda.synchronize()
+    for key in ("spatial", "temporal", "importance", "ratio"):
+        assert rel_err(to_host(g[key]), o[key]) <= TIGHT_TOL, key
+    np.testing.assert_array_equal(to_host(g["k"]), o["k"])
+    # a uniform frame of bf16 tokens whose fp32 mean is a rounded multiple of the token
+    xb = W.f32_to_bf16_bits(np.tile(np.random.default_rng(53).standard_normal((1, 64)).astype(np.float32), (7, 1)))
+    ob = orc.score_frames(xb, [0, 1], 7)
+    gb = sv.sharpv_score_frames(to_dev(xb), torch.tensor([0, 1], dtype=torch.int32, device=dev), 1, 7,
+                                want_spatial=True)
+    torch.cuda.synchronize()
+    assert rel_err(to_host(gb["spatial"]), ob["spatial"]) <= TIGHT_TOL
+    # stage two with zero hidden rows and a sequence without visual tokens
+    hid = np.random.default_rng(54).standard_normal((10, 16)).astype(np.float32)
+    vis = hid[2:6].copy()
+    hid[3] = 0.0
+    so, vb, vc, vo = [0, 8, 10], [2, 0], [4, 0], [0, 4]
+    oc = orc.kv_calibrate_prune(hid, vis, so, vb, vc, vo, M=0.5)
+    t32 = lambda a: torch.tensor(a, dtype=torch.int32, device=dev)
+    gc = sv.sharpv_kv_calibrate_prune(to_dev(hid), to_dev(vis), t32(so), t32(vb), t32(vc), t32(vo), 10, M=0.5,
+                                      want_mean_cos=True)
+    torch.cuda.synchronize()
+    n = int(gc["kept_seq_offsets"][-1].item())
+    np.testing.assert_array_equal(to_host(gc["kept_pos"])[:n], oc["kept_pos"])
+    np.testing.assert_array_equal(to_host(gc["kept_seq_offsets"]), oc["kept_seq_offsets"])
+    assert rel_err(to_host(gc["cos"]), oc["cos"]) <= TIGHT_TOL
+    assert to_host(gc["mean_cos"])[1] == 0.0
+
+
+def test_run_to_run_bit_reproducible():
+    wl, dw = _case("small_ragged")
+    F, f = wl.total_frames, wl.f
+    a = sv.sharpv_score_frames(dw.tokens, dw.video_frame_offsets, F, f, want_spatial=True, want_temporal=True)
+    b = sv.sharpv_score_frames(dw.tokens, dw.video_frame_offsets, F, f, want_spatial=True, want_temporal=True)
+    torch.cuda.synchronize()
+    for key in a:
+        assert torch.equal(a[key], b[key]), key
+
+
+def test_strided_token_rows():
+    """Row stride larger than d (tokens embedded in a wider buffer)."""
+    wl, dw = _case("tiny")
+    F, f, d = wl.total_frames, wl.f, wl.d
+    wide = torch.zeros((wl.n_visual, d + 64), dtype=dw.tokens.dtype, device="cuda")
+    wide[:, :d] = dw.tokens
+    a = sv.sharpv_score_frames(dw.tokens, dw.video_frame_offsets, F, f)
+    b = sv.sharpv_score_frames(wide[:, :d], dw.video_frame_offsets, F, f)
+    torch.cuda.synchronize()
+    assert torch.equal(a["importance"], b["importance"]) and torch.equal(a["k"], b["k"])
+    sa = sv.sharpv_select_tokens(a["importance"], a["k"], F, f, tokens=dw.tokens)
+    sb = sv.sharpv_select_tokens(b["importance"], b["k"], F, f, tokens=wide[:, :d])
+    torch.cuda.synchronize()
+    n = int(sa["num_kept"].item())
+    assert torch.equal(sa["tokens"][:n], sb["tokens"][:n])
