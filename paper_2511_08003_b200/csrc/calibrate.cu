@@ -147,7 +147,7 @@ extern "C" size_t sharpv_kv_calibrate_prune_workspace_bytes(int64_t total_seq_to
     return ws_flags_bytes(total_seq_tokens) + align_up((size_t)num_chunks(total_seq_tokens) * 4, 256);
 }
 
-extern "C" sharpv_status sharpv_kv_calibrate_prune(
+static sharpv_status calibrate_impl(
     const void* hidden, int64_t ld_hidden, const void* visual, int64_t ld_visual, sharpv_dtype dtype,
     int32_t d, int32_t num_seqs, const int32_t* seq_offsets, const int32_t* vis_begin,
     const int32_t* vis_count, const int32_t* vis_offsets, int64_t total_seq_tokens, int64_t total_visual,
@@ -194,4 +194,16 @@ extern "C" sharpv_status sharpv_kv_calibrate_prune(
     if (out_mean_cos)
         mean_cos_kernel<<<num_seqs, 256, 0, stream>>>(out_cos, vis_count, vis_offsets, total_visual, out_mean_cos);
     return launch_status();
+}
+
+extern "C" sharpv_status sharpv_kv_calibrate_prune(
+    const void* hidden, int64_t ld_hidden, const void* visual, int64_t ld_visual, sharpv_dtype dtype,
+    int32_t d, int32_t num_seqs, const int32_t* seq_offsets, const int32_t* vis_begin,
+    const int32_t* vis_count, const int32_t* vis_offsets, int64_t total_seq_tokens, int64_t total_visual,
+    float M, float* out_cos, float* out_mean_cos, int32_t* out_kept_pos, int32_t* out_kept_seq_offsets,
+    int64_t capacity, void* workspace, size_t workspace_bytes, int32_t* status_word, void* cuda_stream) {
+    return calibrate_impl(hidden, ld_hidden, visual, ld_visual, dtype, d, num_seqs, seq_offsets, vis_begin,
+                          vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, out_mean_cos,
+                          out_kept_pos, out_kept_seq_offsets, capacity, workspace, workspace_bytes, status_word,
+                          cuda_stream);
 }
