@@ -167,6 +167,42 @@ sharpv_status sharpv_kv_calibrate_prune(
     void* workspace, size_t workspace_bytes, int32_t* status_word, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Allocation-free variant of sharpv_kv_calibrate_prune.  (No counterpart in the paper: this is a
+ * packaging of the same operation for hosts that cannot provide scratch memory.)
+ *
+ * Some callers have no way to hand over a workspace: a serving engine that gave all free device
+ * memory to its own K/V-cache pool at start-up and can neither carve a temporary out of it nor
+ * risk a cudaMalloc that fails or stalls every stream; a plug-in that only receives the tensors
+ * of the operation and has no allocator handle; a process running under a fixed memory budget
+ * where any late allocation is refused.  For them the keep flags and per-chunk counts live in
+ * a fixed array inside the library's device image, sized for at most
+ * SHARPV_NOALLOC_MAX_SEQ_TOKENS packed positions (about 260 KB, resident on every GPU that
+ * loads the library until the process exits).
+ *
+ * Arguments, outputs and results are those of sharpv_kv_calibrate_prune without `workspace` and
+ * `workspace_bytes`.  The call performs no cudaMalloc / cudaFree and calls no allocating library
+ * routine.  total_seq_tokens > SHARPV_NOALLOC_MAX_SEQ_TOKENS returns SHARPV_ERR_UNSUPPORTED and
+ * launches nothing.
+ * The first call on each device looks up the device address of the array (one runtime query, made
+ * with that device current); make that first call outside any stream capture.  All calls on a
+ * device share the one array: two calls whose kernels may overlap on the GPU (different streams
+ * without ordering between them) race on it and must be serialised by the caller.  The array
+ * keeps the previous call's contents; every entry that a call reads is written by that call
+ * first, so no clearing is needed between calls.
+ */
+#define SHARPV_NOALLOC_MAX_SEQ_TOKENS 262144
+
+sharpv_status sharpv_kv_calibrate_prune_noalloc(
+    const void* hidden, int64_t ld_hidden, const void* visual, int64_t ld_visual,
+    sharpv_dtype dtype, int32_t d,
+    int32_t num_seqs, const int32_t* seq_offsets, const int32_t* vis_begin,
+    const int32_t* vis_count, const int32_t* vis_offsets,
+    int64_t total_seq_tokens, int64_t total_visual, float M,
+    float* out_cos, float* out_mean_cos,
+    int32_t* out_kept_pos, int32_t* out_kept_seq_offsets, int64_t capacity,
+    int32_t* status_word, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
  * Stage two (b): K/V compaction.  Section 3.2.3: the discarded tokens' K/V is dropped so that
  * decoding only reads what was retained (Section 1, "retain visual tokens for subsequent
  * generation steps").

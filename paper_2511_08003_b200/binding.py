@@ -54,8 +54,11 @@ EXPORTS = (
     "sharpv_score_frames_workspace_bytes", "sharpv_score_frames",
     "sharpv_select_tokens_workspace_bytes", "sharpv_select_tokens", "sharpv_select_tokens_threshold",
     "sharpv_kv_calibrate_prune_workspace_bytes", "sharpv_kv_calibrate_prune",
+    "sharpv_kv_calibrate_prune_noalloc",
     "sharpv_kv_compact",
 )
+
+NOALLOC_MAX_SEQ_TOKENS = 262144
 
 
 def lib_path() -> str:
@@ -93,6 +96,9 @@ def lib():
     L.sharpv_kv_calibrate_prune.restype = C.c_int
     L.sharpv_kv_calibrate_prune.argtypes = [vp, i64, vp, i64, C.c_int, i32, i32, vp, vp, vp, vp, i64, i64, f32,
                                             vp, vp, vp, vp, i64, vp, sz, vp, vp]
+    L.sharpv_kv_calibrate_prune_noalloc.restype = C.c_int
+    L.sharpv_kv_calibrate_prune_noalloc.argtypes = [vp, i64, vp, i64, C.c_int, i32, i32, vp, vp, vp, vp, i64, i64,
+                                                    f32, vp, vp, vp, vp, i64, vp, vp]
     L.sharpv_kv_compact.restype = C.c_int
     L.sharpv_kv_compact.argtypes = [vp, C.POINTER(KVLayout), vp, C.POINTER(KVLayout), i32, i32, vp, vp, i32, i64,
                                     vp, vp]
@@ -250,12 +256,8 @@ def sharpv_kv_calibrate_prune_workspace_bytes(total_seq_tokens: int, num_seqs: i
     return int(lib().sharpv_kv_calibrate_prune_workspace_bytes(total_seq_tokens, num_seqs))
 
 
-def sharpv_kv_calibrate_prune(hidden: torch.Tensor, visual: torch.Tensor, seq_offsets: torch.Tensor,
-                              vis_begin: torch.Tensor, vis_count: torch.Tensor, vis_offsets: torch.Tensor,
-                              total_seq_tokens: int, M: float = 0.2, capacity: Optional[int] = None,
-                              want_mean_cos: bool = False, out=None, workspace=None, status_word=None,
-                              stream=None):
-    """Self-calibration of stage two.  Returns dict(cos, kept_pos, kept_seq_offsets[, mean_cos])."""
+def _calibrate(fn_name, hidden, visual, seq_offsets, vis_begin, vis_count, vis_offsets, total_seq_tokens, M,
+               capacity, want_mean_cos, out, workspace, status_word, stream):
     ldh, ldv = _rows(hidden, "hidden"), _rows(visual, "visual")
     if hidden.dtype != visual.dtype or hidden.shape[1] != visual.shape[1]:
         raise ValueError("hidden and visual must share dtype and feature size")
@@ -273,17 +275,43 @@ def sharpv_kv_calibrate_prune(hidden: torch.Tensor, visual: torch.Tensor, seq_of
         out["kept_seq_offsets"] = torch.empty(B + 1, dtype=torch.int32, device=dev)
     if want_mean_cos and "mean_cos" not in out:
         out["mean_cos"] = torch.empty(B, dtype=torch.float32, device=dev)
-    ws = _workspace(workspace, sharpv_kv_calibrate_prune_workspace_bytes(total_seq_tokens, B), dev)
-    rc = lib().sharpv_kv_calibrate_prune(
-        _dev(hidden, "hidden"), ldh, _dev(visual, "visual"), ldv, _dtype_code(hidden), hidden.shape[1], B,
-        _dev(seq_offsets, "seq_offsets", torch.int32), _dev(vis_begin, "vis_begin", torch.int32),
-        _dev(vis_count, "vis_count", torch.int32), _dev(vis_offsets, "vis_offsets", torch.int32),
-        total_seq_tokens, total_visual, float(M), _dev(out["cos"], "cos", torch.float32),
-        _dev(out.get("mean_cos"), "mean_cos", torch.float32), _dev(out["kept_pos"], "kept_pos", torch.int32),
-        _dev(out["kept_seq_offsets"], "kept_seq_offsets", torch.int32), capacity, ws.data_ptr(), ws.numel(),
-        _dev(status_word, "status_word", torch.int32), _stream(stream))
-    _check("sharpv_kv_calibrate_prune", rc)
+    head = (_dev(hidden, "hidden"), ldh, _dev(visual, "visual"), ldv, _dtype_code(hidden), hidden.shape[1], B,
+            _dev(seq_offsets, "seq_offsets", torch.int32), _dev(vis_begin, "vis_begin", torch.int32),
+            _dev(vis_count, "vis_count", torch.int32), _dev(vis_offsets, "vis_offsets", torch.int32),
+            total_seq_tokens, total_visual, float(M), _dev(out["cos"], "cos", torch.float32),
+            _dev(out.get("mean_cos"), "mean_cos", torch.float32), _dev(out["kept_pos"], "kept_pos", torch.int32),
+            _dev(out["kept_seq_offsets"], "kept_seq_offsets", torch.int32), capacity)
+    tail = (_dev(status_word, "status_word", torch.int32), _stream(stream))
+    if fn_name == "sharpv_kv_calibrate_prune":
+        ws = _workspace(workspace, sharpv_kv_calibrate_prune_workspace_bytes(total_seq_tokens, B), dev)
+        rc = lib().sharpv_kv_calibrate_prune(*head, ws.data_ptr(), ws.numel(), *tail)
+    else:
+        rc = lib().sharpv_kv_calibrate_prune_noalloc(*head, *tail)
+    _check(fn_name, rc)
     return out
+
+
+def sharpv_kv_calibrate_prune(hidden: torch.Tensor, visual: torch.Tensor, seq_offsets: torch.Tensor,
+                              vis_begin: torch.Tensor, vis_count: torch.Tensor, vis_offsets: torch.Tensor,
+                              total_seq_tokens: int, M: float = 0.2, capacity: Optional[int] = None,
+                              want_mean_cos: bool = False, out=None, workspace=None, status_word=None,
+                              stream=None):
+    """Self-calibration of stage two.  Returns dict(cos, kept_pos, kept_seq_offsets[, mean_cos])."""
+    return _calibrate("sharpv_kv_calibrate_prune", hidden, visual, seq_offsets, vis_begin, vis_count, vis_offsets,
+                      total_seq_tokens, M, capacity, want_mean_cos, out, workspace, status_word, stream)
+
+
+def sharpv_kv_calibrate_prune_noalloc(hidden: torch.Tensor, visual: torch.Tensor, seq_offsets: torch.Tensor,
+                                      vis_begin: torch.Tensor, vis_count: torch.Tensor,
+                                      vis_offsets: torch.Tensor, total_seq_tokens: int, M: float = 0.2,
+                                      capacity: Optional[int] = None, want_mean_cos: bool = False, out=None,
+                                      status_word=None, stream=None):
+    """Same operation and outputs as sharpv_kv_calibrate_prune for hosts that cannot supply scratch
+    memory: the library's built-in scratch array is used (at most NOALLOC_MAX_SEQ_TOKENS packed positions).
+    The library call itself allocates nothing; pass every output in `out` if this wrapper must not
+    allocate either.  Calls on one device share the scratch and must not overlap on the GPU."""
+    return _calibrate("sharpv_kv_calibrate_prune_noalloc", hidden, visual, seq_offsets, vis_begin, vis_count,
+                      vis_offsets, total_seq_tokens, M, capacity, want_mean_cos, out, None, status_word, stream)
 
 
 def sharpv_kv_compact(kv_src: torch.Tensor, kv_dst: torch.Tensor, kept_pos: torch.Tensor,

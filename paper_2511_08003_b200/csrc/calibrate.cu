@@ -7,6 +7,8 @@
 //   write_kept_kernel     same chunks: chunk base = sum of earlier chunk counts, local scan,
 //                         ascending kept positions, per-sequence offsets, capacity check
 //   mean_cos_kernel       (optional) fixed-order mean of the cosines of each sequence
+#include <mutex>
+
 #include "common.cuh"
 
 namespace sharpv {
@@ -206,4 +208,59 @@ extern "C" sharpv_status sharpv_kv_calibrate_prune(
                           vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, out_mean_cos,
                           out_kept_pos, out_kept_seq_offsets, capacity, workspace, workspace_bytes, status_word,
                           cuda_stream);
+}
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free variant: the scratch lives in a file-scope device array
+// ---------------------------------------------------------------------------------------
+namespace {
+
+constexpr int64_t kNoAllocMaxTokens = SHARPV_NOALLOC_MAX_SEQ_TOKENS;
+constexpr size_t kNoAllocScratchBytes =
+    ((size_t)kNoAllocMaxTokens + 255) / 256 * 256 +                                   // keep flags
+    (((size_t)(kNoAllocMaxTokens + kChunk - 1) / kChunk) * 4 + 255) / 256 * 256;      // per-chunk counts
+
+// Held by every GPU that loads this library until the process exits (about 260 KB).
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+void* g_noalloc_ptr[kMaxDevices] = {};     // device address of g_noalloc_scratch, per device
+
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not an address a kernel can
+// use: the device address has to be asked for, once per device, with that device current.
+sharpv_status noalloc_scratch(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SHARPV_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return SHARPV_ERR_CUDA;
+        }
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = g_noalloc_ptr[dev];
+    return SHARPV_OK;
+}
+
+}  // namespace
+
+extern "C" sharpv_status sharpv_kv_calibrate_prune_noalloc(
+    const void* hidden, int64_t ld_hidden, const void* visual, int64_t ld_visual, sharpv_dtype dtype,
+    int32_t d, int32_t num_seqs, const int32_t* seq_offsets, const int32_t* vis_begin,
+    const int32_t* vis_count, const int32_t* vis_offsets, int64_t total_seq_tokens, int64_t total_visual,
+    float M, float* out_cos, float* out_mean_cos, int32_t* out_kept_pos, int32_t* out_kept_seq_offsets,
+    int64_t capacity, int32_t* status_word, void* cuda_stream) {
+    if (total_seq_tokens > kNoAllocMaxTokens) return SHARPV_ERR_UNSUPPORTED;
+    void* scratch = nullptr;
+    const sharpv_status st = noalloc_scratch(&scratch);
+    if (st != SHARPV_OK) return st;
+    // Every flag and every chunk count below total_seq_tokens is rewritten by the kernels before it
+    // is read, so nothing left over from the previous call has to be cleared.
+    return calibrate_impl(hidden, ld_hidden, visual, ld_visual, dtype, d, num_seqs, seq_offsets, vis_begin,
+                          vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, out_mean_cos,
+                          out_kept_pos, out_kept_seq_offsets, capacity, scratch, kNoAllocScratchBytes,
+                          status_word, cuda_stream);
 }
