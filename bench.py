@@ -15,9 +15,7 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
 import sys
-import tempfile
 import time
 
 import numpy as np
@@ -39,7 +37,7 @@ NCU_TRAFFIC_BYTES = {}
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="onevision_7b", choices=list(W.PRESETS))
     ap.add_argument("--impl", default="sharpv", choices=["sharpv", "reference"])
@@ -144,54 +142,54 @@ def run_reference(args):
 
 # ------------------------------------------------------------------------------------- clocks
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and throttle reasons of one GPU from a thread while the timed region runs
+    (NVML, read-only queries)."""
 
-    def __init__(self, index):
-        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        self.proc = None
+    REASONS = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40}
+
+    def __init__(self, index, period_s=0.005, pci_bus_id=None):
+        import threading
+        self.samples, self.reason_bits, self.max_mhz = [], 0, None
+        self._stop = threading.Event()
+        self._thread = None
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+            import pynvml
+            pynvml.nvmlInit()
+            self._nvml = pynvml
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByPciBusId(pci_bus_id.encode()) if pci_bus_id else None
+            except Exception:
+                self._h = None
+            if self._h is None:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
         except Exception:
-            self.proc = None
+            self._nvml = None
+            return
+        self._period = period_s
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+
+    def _run(self):
+        nv = self._nvml
+        while not self._stop.is_set():
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+            except Exception:
+                pass
+            self._stop.wait(self._period)
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
-        if self.proc is None:
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": []}
+        if self._thread is None:
             return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        self.tmp.flush()
-        self.tmp.seek(0)
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.tmp.read().splitlines():
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 7:
-                continue
-            try:
-                sm.append(float(parts[0]))
-                mx.append(float(parts[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, parts[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        try:
-            os.unlink(self.tmp.name)
-        except OSError:
-            pass
-        if sm:
-            out["sm_mhz"] = statistics.median(sm)
-            out["sm_max_mhz"] = max(mx)
-            out["samples"] = len(sm)
-        out["reasons"] = sorted(reasons)
+        self._stop.set()
+        self._thread.join(timeout=2)
+        if self.samples:
+            out["sm_mhz"] = statistics.median(self.samples)
+            out["samples"] = len(self.samples)
+        out["reasons"] = sorted(n for n, bit in self.REASONS.items() if self.reason_bits & bit)
         return out
 
 
@@ -273,13 +271,9 @@ def run_sharpv(args):
     stages = [("score", stage_score), ("select", stage_select), ("calibrate", stage_calibrate),
               ("compact", stage_compact)]
 
-    def step(events=None):
-        for i, (_, fn) in enumerate(stages):
-            if events is not None:
-                events[i].record(stream)
+    def step():
+        for _, fn in stages:
             fn()
-        if events is not None:
-            events[len(stages)].record(stream)
 
     def barrier():
         torch.cuda.synchronize()
@@ -287,7 +281,8 @@ def run_sharpv(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    W_ = max(args.warmup, 3)
+    for _ in range(W_):
         flush.zero_()
         step()
     torch.cuda.synchronize()
@@ -295,20 +290,56 @@ def run_sharpv(args):
     t_keep = int(o_cal["kept_seq_offsets"][-1].item())
     assert int(status.item()) == 0, "device status word set"
 
-    # ---- timed region: K steps, device-timed, L2 flushed between steps (flush not timed)
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)] for _ in range(args.steps)]
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    # The library calls only enqueue kernels (no allocation, no sync), so one step is captured
+    # into a CUDA graph and replayed: the GPU never waits for the Python caller.
+    graph = torch.cuda.CUDAGraph()
+    cap_stream = torch.cuda.Stream()
+    cap_stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(cap_stream):
+        with torch.cuda.graph(graph, stream=cap_stream):
+            step()
+    torch.cuda.synchronize()
+    for _ in range(W_):
+        flush.zero_()
+        graph.replay()
+    torch.cuda.synchronize()
+
+    # ---- timed region: K graph replays, device-timed; the L2 flush before each is not timed
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    try:
+        pr = torch.cuda.get_device_properties(dev)
+        bus = f"{pr.pci_domain_id:08x}:{pr.pci_bus_id:02x}:{pr.pci_device_id:02x}.0"
+    except Exception:
+        bus = None
+    sampler = ClockSampler(local_rank, pci_bus_id=bus) if rank == 0 else None
     barrier()
     wall0 = time.perf_counter()
     for s in range(args.steps):
         flush.zero_()
-        step(ev[s])
+        ev[s][0].record(stream)
+        graph.replay()
+        ev[s][1].record(stream)
     barrier()
     wall = time.perf_counter() - wall0
-    clocks = sampler.stop() if sampler else None
-    step_ms = [e[0].elapsed_time(e[-1]) for e in ev]
-    stage_ms = {name: statistics.fmean(e[i].elapsed_time(e[i + 1]) for e in ev) for i, (name, _) in enumerate(stages)}
+    step_ms = [a.elapsed_time(b) for a, b in ev]
     total_ms = sum(step_ms)
+
+    # ---- per-stage launch durations, each from a cold L2 (same events, same stream, same region
+    # of the run; the flush kernel is long enough for the host to queue the stage behind it)
+    stage_steps = max(5, min(args.steps, 50))
+    stage_ms = {}
+    for name, fn in stages:
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(stage_steps)]
+        for a, b in evs:
+            flush.zero_()
+            a.record(stream)
+            fn()
+            b.record(stream)
+        torch.cuda.synchronize()
+        stage_ms[name] = statistics.fmean(a.elapsed_time(b) for a, b in evs)
+    clocks = sampler.stop() if sampler else None
+
     if world > 1:
         t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -388,15 +419,18 @@ def run_sharpv(args):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": W_, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "frames": F, "tokens_per_frame": f, "d": d, "storage": wl.dtype,
                    "visual_tokens": NV, "seq_tokens": T, "kv": list(wl.kv_shape()), "M": args.M, "w": args.w,
                    "kept_stage_one": n_keep, "kept_stage_two": t_keep,
-                   "l2": "512 MB buffer overwritten before every timed step (not timed); each step also moves "
-                         "more K/V than the 126 MB L2 holds"},
+                   "launch": "one CUDA graph replay per step",
+                   "l2": "512 MB buffer overwritten before every timed step and before every per-kernel "
+                         "launch (not timed); each step also moves more K/V than the 126 MB L2 holds"},
         "kv_compaction_GBps": kernels["compact"]["GBps"],
         "roofline": roofline, "kernels": kernels,
+        "step_ms": {"min": round(min(step_ms), 5), "median": round(statistics.median(step_ms), 5),
+                    "max": round(max(step_ms), 5)},
         "cpu_baseline": cpu,
         "e2e": {"value": world * NV / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

@@ -187,8 +187,9 @@ sharpv_status sharpv_kv_calibrate_prune(
  * with that device current); make that first call outside any stream capture.  All calls on a
  * device share the one array: two calls whose kernels may overlap on the GPU (different streams
  * without ordering between them) race on it and must be serialised by the caller.  The array
- * keeps the previous call's contents; every entry that a call reads is written by that call
- * first, so no clearing is needed between calls.
+ * keeps the previous call's contents; each call clears the counters it accumulates into (on the
+ * stream, before its kernels) and overwrites every flag before reading it, so the caller never has
+ * to clear anything between calls.
  */
 #define SHARPV_NOALLOC_MAX_SEQ_TOKENS 262144
 

@@ -2,8 +2,8 @@
 // followed by the compaction of the keep flags into ascending kept positions.
 //
 // Kernels:
-//   calibrate_cos_kernel  one warp per packed position: cos(hidden row, visual row), keep flag;
-//                         each CTA also writes how many of its positions survive
+//   calibrate_cos_kernel  one warp per packed position: cos(hidden row, visual row), keep flag,
+//                         and an integer count of survivors per chunk of 256 positions
 //   write_kept_kernel     same chunks: chunk base = sum of earlier chunk counts, local scan,
 //                         ascending kept positions, per-sequence offsets, capacity check
 //   mean_cos_kernel       (optional) fixed-order mean of the cosines of each sequence
@@ -14,10 +14,12 @@
 namespace sharpv {
 namespace {
 
-constexpr int kChunk = 256;             // packed positions per CTA (8 warps x 32 positions)
+constexpr int kChunk = 256;             // packed positions per chunk of the flag scan
 
 __host__ __device__ inline size_t ws_flags_bytes(int64_t T) { return ((size_t)T + 255) / 256 * 256; }
 __host__ __device__ inline int64_t num_chunks(int64_t T) { return (T + kChunk - 1) / kChunk; }
+
+constexpr int kRowsPerCta = 8;          // one packed position per warp
 
 template <int DT>
 __global__ void __launch_bounds__(256)
@@ -30,26 +32,31 @@ calibrate_cos_kernel(const char* __restrict__ hidden, int64_t hidden_row_bytes,
                      int32_t* __restrict__ chunk_counts) {
     using E = Elem<DT>;
     constexpr int P = E::kPerVec;
-    __shared__ int warp_kept[8];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t chunk_base = (int64_t)blockIdx.x * kChunk;
-    int kept_here = 0;
-    for (int q = 0; q < kChunk / 8; ++q) {
-        const int64_t p = chunk_base + warp * (kChunk / 8) + q;
-        if (p >= T) break;
-        const int b = upper_segment(seq_offsets, num_seqs, (int)p);
-        const int64_t local = p - __ldg(seq_offsets + b) - __ldg(vis_begin + b);
-        int keep = 1;
-        if (local >= 0 && local < __ldg(vis_count + b)) {
-            const int64_t vrow = (int64_t)__ldg(vis_offsets + b) + local;
-            if (vrow < total_visual) {
-                const char* ph = hidden + p * hidden_row_bytes;
-                const char* pv = visual + vrow * visual_row_bytes;
-                float shh = 0.f, svv = 0.f, shv = 0.f;
-                for (int v = lane; v < nvec; v += 32) {
+    const int64_t p = (int64_t)blockIdx.x * kRowsPerCta + warp;
+    if (p >= T) return;
+    const int b = upper_segment(seq_offsets, num_seqs, (int)p);
+    const int64_t local = p - __ldg(seq_offsets + b) - __ldg(vis_begin + b);
+    int keep = 1;
+    if (local >= 0 && local < __ldg(vis_count + b)) {
+        const int64_t vrow = (int64_t)__ldg(vis_offsets + b) + local;
+        if (vrow < total_visual) {
+            const char* ph = hidden + p * hidden_row_bytes;
+            const char* pv = visual + vrow * visual_row_bytes;
+            float shh = 0.f, svv = 0.f, shv = 0.f;
+            int v = lane;
+            for (; v + 96 < nvec; v += 128) {           // 8 independent 128-bit loads in flight
+                uint4 rh[4], rv[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    rh[u] = ld_stream(ph + (int64_t)(v + 32 * u) * 16);
+                    rv[u] = ld_stream(pv + (int64_t)(v + 32 * u) * 16);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
                     float h[P], x[P];
-                    E::widen(ld_stream(ph + (int64_t)v * 16), h);
-                    E::widen(ld_stream(pv + (int64_t)v * 16), x);
+                    E::widen(rh[u], h);
+                    E::widen(rv[u], x);
 #pragma unroll
                     for (int j = 0; j < P; ++j) {
                         shh = fmaf(h[j], h[j], shh);
@@ -57,23 +64,28 @@ calibrate_cos_kernel(const char* __restrict__ hidden, int64_t hidden_row_bytes,
                         shv = fmaf(h[j], x[j], shv);
                     }
                 }
-                shh = warp_sum(shh); svv = warp_sum(svv); shv = warp_sum(shv);
-                const float nh = fmaxf(sqrtf(shh), kNormEps), nv = fmaxf(sqrtf(svv), kNormEps);
-                const float c = shv / (nh * nv);
-                keep = c < M ? 0 : 1;                       // Eq. 7: discard iff cos < M
-                if (lane == 0) out_cos[vrow] = c;
             }
-        }
-        if (lane == 0) flags[p] = (uint8_t)keep;
-        kept_here += keep;
-    }
-    if (lane == 0) warp_kept[warp] = kept_here;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int tot = 0;
+            for (; v < nvec; v += 32) {
+                float h[P], x[P];
+                E::widen(ld_stream(ph + (int64_t)v * 16), h);
+                E::widen(ld_stream(pv + (int64_t)v * 16), x);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) tot += warp_kept[i];
-        chunk_counts[blockIdx.x] = tot;
+                for (int j = 0; j < P; ++j) {
+                    shh = fmaf(h[j], h[j], shh);
+                    svv = fmaf(x[j], x[j], svv);
+                    shv = fmaf(h[j], x[j], shv);
+                }
+            }
+            shh = warp_sum(shh); svv = warp_sum(svv); shv = warp_sum(shv);
+            const float nh = fmaxf(sqrtf(shh), kNormEps), nv = fmaxf(sqrtf(svv), kNormEps);
+            const float c = shv / (nh * nv);
+            keep = c < M ? 0 : 1;                       // Eq. 7: discard iff cos < M
+            if (lane == 0) out_cos[vrow] = c;
+        }
+    }
+    if (lane == 0) {
+        flags[p] = (uint8_t)keep;
+        if (keep) atomicAdd(chunk_counts + p / kChunk, 1);     // integer: order does not matter
     }
 }
 
@@ -182,13 +194,17 @@ static sharpv_status calibrate_impl(
     uint8_t* flags = (uint8_t*)workspace;
     int32_t* chunk_counts = (int32_t*)((char*)workspace + ws_flags_bytes(total_seq_tokens));
     const unsigned chunks = (unsigned)num_chunks(total_seq_tokens);
+    const unsigned ctas = (unsigned)((total_seq_tokens + kRowsPerCta - 1) / kRowsPerCta);
     const int nvec = d * eb / 16;
+    // the per-chunk counts are accumulated with atomics and must start at zero
+    if (cudaMemsetAsync(chunk_counts, 0, sizeof(int32_t) * (size_t)chunks, stream) != cudaSuccess)
+        return SHARPV_ERR_CUDA;
     if (dtype == SHARPV_F32)
-        calibrate_cos_kernel<SHARPV_F32><<<chunks, 256, 0, stream>>>(
+        calibrate_cos_kernel<SHARPV_F32><<<ctas, 256, 0, stream>>>(
             (const char*)hidden, ld_hidden * eb, (const char*)visual, ld_visual * eb, nvec, num_seqs, seq_offsets,
             vis_begin, vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, flags, chunk_counts);
     else
-        calibrate_cos_kernel<SHARPV_BF16><<<chunks, 256, 0, stream>>>(
+        calibrate_cos_kernel<SHARPV_BF16><<<ctas, 256, 0, stream>>>(
             (const char*)hidden, ld_hidden * eb, (const char*)visual, ld_visual * eb, nvec, num_seqs, seq_offsets,
             vis_begin, vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, flags, chunk_counts);
     write_kept_kernel<<<chunks, kChunk, 0, stream>>>(flags, chunk_counts, total_seq_tokens, num_seqs, seq_offsets,
@@ -257,8 +273,8 @@ extern "C" sharpv_status sharpv_kv_calibrate_prune_noalloc(
     void* scratch = nullptr;
     const sharpv_status st = noalloc_scratch(&scratch);
     if (st != SHARPV_OK) return st;
-    // Every flag and every chunk count below total_seq_tokens is rewritten by the kernels before it
-    // is read, so nothing left over from the previous call has to be cleared.
+    // Every flag below total_seq_tokens is rewritten before it is read and the chunk counts are
+    // cleared on the stream at the start of each call, so the previous call leaves nothing behind.
     return calibrate_impl(hidden, ld_hidden, visual, ld_visual, dtype, d, num_seqs, seq_offsets, vis_begin,
                           vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, out_mean_cos,
                           out_kept_pos, out_kept_seq_offsets, capacity, scratch, kNoAllocScratchBytes,
