@@ -1,11 +1,13 @@
 // Stage one (a): spatial / temporal dissimilarity scores and the adaptive per-frame budget
 // (Section 3.1.2 - 3.1.3, Eq. 1-6).
 //
-// Three kernels:
+// Shapes that split into 256-byte column slices with frames of up to 208 tokens run in the single
+// fused kernel of score_fused.cu.  Every other shape runs the three kernels below:
 //   frame_mean_kernel   column sums of each frame -> frame mean (fp32), first-frame flags
 //   row_scores_kernel   one warp per token: the row reductions behind S, T and I
 //   frame_budget_kernel one CTA per frame: ||T_t||_2 -> ratio_t, k_t (fixed-order reduction)
-#include "common.cuh"
+#include "score_common.cuh"
+#include "score_fused.cuh"
 
 namespace sharpv {
 namespace {
@@ -38,36 +40,32 @@ frame_mean_kernel(const char* __restrict__ tokens, int64_t row_bytes_ld, int f, 
     }
     if (v >= nvec) return;
     const char* base = tokens + (int64_t)t * f * row_bytes_ld + (int64_t)v * 16;
-    float acc[P];
+    // compensated (Kahan) column sums: the mean stays accurate to about one ulp however long the
+    // frame is, which the spatial score of an almost uniform frame depends on; the kernel is
+    // bandwidth-bound, so the extra adds are free
+    float acc[P], comp[P];
 #pragma unroll
-    for (int j = 0; j < P; ++j) acc[j] = 0.f;
+    for (int j = 0; j < P; ++j) { acc[j] = 0.f; comp[j] = 0.f; }
+    auto add_row = [&](const uint4& r) {
+        float x[P];
+        E::widen(r, x);
+#pragma unroll
+        for (int j = 0; j < P; ++j) {
+            const float y = __fsub_rn(x[j], comp[j]);
+            const float tsum = __fadd_rn(acc[j], y);
+            comp[j] = __fsub_rn(__fsub_rn(tsum, acc[j]), y);
+            acc[j] = tsum;
+        }
+    };
     int i = 0;
     for (; i + 4 <= f; i += 4) {
         uint4 r0 = ld_stream(base + (int64_t)(i + 0) * row_bytes_ld);
         uint4 r1 = ld_stream(base + (int64_t)(i + 1) * row_bytes_ld);
         uint4 r2 = ld_stream(base + (int64_t)(i + 2) * row_bytes_ld);
         uint4 r3 = ld_stream(base + (int64_t)(i + 3) * row_bytes_ld);
-        float x[P];
-        E::widen(r0, x);
-#pragma unroll
-        for (int j = 0; j < P; ++j) acc[j] += x[j];
-        E::widen(r1, x);
-#pragma unroll
-        for (int j = 0; j < P; ++j) acc[j] += x[j];
-        E::widen(r2, x);
-#pragma unroll
-        for (int j = 0; j < P; ++j) acc[j] += x[j];
-        E::widen(r3, x);
-#pragma unroll
-        for (int j = 0; j < P; ++j) acc[j] += x[j];
+        add_row(r0); add_row(r1); add_row(r2); add_row(r3);
     }
-    for (; i < f; ++i) {
-        uint4 r0 = ld_stream(base + (int64_t)i * row_bytes_ld);
-        float x[P];
-        E::widen(r0, x);
-#pragma unroll
-        for (int j = 0; j < P; ++j) acc[j] += x[j];
-    }
+    for (; i < f; ++i) add_row(ld_stream(base + (int64_t)i * row_bytes_ld));
     const float ff = (float)f;
     float* out = mean + (int64_t)t * d + (int64_t)v * P;
 #pragma unroll
@@ -76,28 +74,6 @@ frame_mean_kernel(const char* __restrict__ tokens, int64_t row_bytes_ld, int f, 
         *reinterpret_cast<float4*>(out + j) = o;
     }
 }
-
-// ---------------------------------------------------------------------------------------
-// Dissim from row reductions.
-//   ||a^ - b^||^2 = (||a-b||^2 - (||a|| - ||b||)^2) / (||a|| ||b||)
-// is algebraically 2 - 2 cos but has no cancellation for nearly parallel rows and is exactly
-// zero for identical rows.  Rows that are nearly parallel without being close (b ~ alpha a,
-// or a token next to a mean of identical tokens) are re-evaluated by the caller from the
-// normalised rows themselves.
-// ---------------------------------------------------------------------------------------
-__device__ __forceinline__ float dissim_sq_from_sums(float saa, float sbb, float sdd) {
-    const float na = sqrtf(saa), nb = sqrtf(sbb);
-    if (na >= kNormEps && nb >= kNormEps) {
-        const float dn = na - nb;
-        return fmaxf(sdd - dn * dn, 0.f) / (na * nb);
-    }
-    // at least one (near-)zero vector: v^ = v / max(||v||, eps)
-    const float ca = fmaxf(na, kNormEps), cb = fmaxf(nb, kNormEps);
-    const float sab = 0.5f * (saa + sbb - sdd);
-    return fmaxf(saa / (ca * ca) + sbb / (cb * cb) - 2.f * sab / (ca * cb), 0.f);
-}
-
-constexpr float kRefineBelow = 1e-2f;   // squared Dissim under which the exact form is used
 
 template <int DT>
 __global__ void __launch_bounds__(256)
@@ -157,64 +133,19 @@ row_scores_kernel(const char* __restrict__ tokens, int64_t row_bytes_ld, int f, 
         const float ia = 1.f / na;
         const float im = 1.f / fmaxf(sqrtf(smm), kNormEps);
         const float ib = 1.f / fmaxf(sqrtf(sbb), kNormEps);
-        float es = 0.f, et = 0.f;
-        for (int v = lane; v < nvec; v += 32) {
-            float a[P], b[P], m[P];
-            E::widen(ld_cached(pa + (int64_t)v * 16), a);
-            if (refine_s) {
-#pragma unroll
-                for (int j = 0; j < P; j += 4) {
-                    float4 q = __ldg(reinterpret_cast<const float4*>(pm + (int64_t)v * P + j));
-                    m[j] = q.x; m[j + 1] = q.y; m[j + 2] = q.z; m[j + 3] = q.w;
-                }
-#pragma unroll
-                for (int j = 0; j < P; ++j) {
-                    const float df = fmaf(a[j], ia, -m[j] * im);
-                    es = fmaf(df, df, es);
-                }
-            }
-            if (refine_t) {
-                E::widen(ld_cached(pb + (int64_t)v * 16), b);
-#pragma unroll
-                for (int j = 0; j < P; ++j) {
-                    const float df = fmaf(a[j], ia, -b[j] * ib);
-                    et = fmaf(df, df, et);
-                }
-            }
-        }
-        es = warp_sum(es); et = warp_sum(et);
+        float es, et;
+        refine_row<DT>(pa, pb, pm, nvec, lane, refine_s, refine_t, ia, ib, im, es, et);
         if (refine_s) s2 = es;
         if (refine_t) t2 = et;
     }
 
-    float S, T;
-    if (one_minus_cos) {            // 1 - cos = Dissim^2 / 2
-        S = 0.5f * s2;
-        T = is_first ? S : 0.5f * t2;
-    } else {
-        S = sqrtf(s2);
-        T = is_first ? S : sqrtf(t2);
-    }
+    float S, T, I;
+    scores_from_sq(s2, t2, is_first, one_minus_cos, w, S, T, I);
     if (lane == 0) {
-        out_I[row] = fmaf(w, S, T);
+        out_I[row] = I;
         if (out_S) out_S[row] = S;
         out_T[row] = T;
     }
-}
-
-// ---------------------------------------------------------------------------------------
-// per-frame budget: ratio_t = ||T_t||_2 / (2 sqrt(f)), k_t = clamp(round(ratio_t f))
-// ---------------------------------------------------------------------------------------
-__device__ __forceinline__ int budget_from_ratio(float r, int f, int round_mode, int min_keep) {
-    const float x = r * (float)f;
-    float y;
-    if (round_mode == SHARPV_ROUND_FLOOR) y = floorf(x);
-    else if (round_mode == SHARPV_ROUND_NEAREST) y = floorf(x + 0.5f);
-    else y = ceilf(x);
-    int k = (int)y;
-    k = max(k, min_keep);
-    k = min(k, f);
-    return max(k, 0);
 }
 
 __global__ void __launch_bounds__(256)
@@ -235,7 +166,7 @@ frame_budget_kernel(const float* __restrict__ temporal, int f, int round_mode, i
         float tot = 0.f;
 #pragma unroll
         for (int i = 0; i < 8; ++i) tot += part[i];
-        const float r = sqrtf(tot) / (2.f * sqrtf((float)f));
+        const float r = ratio_from_sumsq(tot, f);
         out_ratio[t] = r;
         out_k[t] = budget_from_ratio(r, f, round_mode, min_keep);
     }
@@ -269,7 +200,10 @@ using namespace sharpv;
 
 extern "C" size_t sharpv_score_frames_workspace_bytes(int32_t total_frames, int32_t f, int32_t d) {
     if (total_frames <= 0 || f <= 0 || d <= 0) return 256;
-    return ws_mean_bytes(total_frames, d) + ws_temporal_bytes(total_frames, f) + ws_first_bytes(total_frames);
+    const size_t generic =
+        ws_mean_bytes(total_frames, d) + ws_temporal_bytes(total_frames, f) + ws_first_bytes(total_frames);
+    const size_t fused = fused_score_workspace_bytes(total_frames, f, d);
+    return generic > fused ? generic : fused;
 }
 
 extern "C" sharpv_status sharpv_score_frames(
@@ -278,7 +212,6 @@ extern "C" sharpv_status sharpv_score_frames(
     sharpv_dissim_kind dissim_kind, sharpv_round round_mode, int32_t min_keep, float* out_importance,
     float* out_spatial, float* out_temporal, float* out_ratio, int32_t* out_k, void* workspace,
     size_t workspace_bytes, int32_t* status_word, void* cuda_stream) {
-    (void)status_word;
     if (!dtype_ok(dtype)) return SHARPV_ERR_UNSUPPORTED;
     if (num_videos < 1 || total_frames < 0 || f < 1 || d < 1 || min_keep < 0 || ld_tokens < d)
         return SHARPV_ERR_INVALID_ARG;
@@ -293,13 +226,24 @@ extern "C" sharpv_status sharpv_score_frames(
         return SHARPV_ERR_UNSUPPORTED;
     if (workspace_bytes < sharpv_score_frames_workspace_bytes(total_frames, f, d)) return SHARPV_ERR_WORKSPACE;
 
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const int omc = dissim_kind == SHARPV_ONE_MINUS_COS;
+    if (fused_score_supported(dtype, f, d)) {
+        FusedScoreArgs a;
+        a.tokens = tokens; a.dtype = dtype; a.ld_tokens = ld_tokens; a.num_videos = num_videos;
+        a.video_frame_offsets = video_frame_offsets; a.F = total_frames; a.f = f; a.d = d; a.w = w;
+        a.one_minus_cos = omc; a.round_mode = (int)round_mode; a.min_keep = min_keep;
+        a.out_I = out_importance; a.out_S = out_spatial; a.out_T = out_temporal; a.out_ratio = out_ratio;
+        a.out_k = out_k; a.workspace = workspace; a.status_word = status_word; a.stream = stream;
+        const sharpv_status st = fused_score_launch(a);
+        if (st != SHARPV_ERR_UNSUPPORTED) return st;      // otherwise: set-up unavailable, use the generic kernels
+    }
+
     ScoreWorkspace ws;
     char* p = (char*)workspace;
     ws.mean = (float*)p;       p += ws_mean_bytes(total_frames, d);
     ws.temporal = (float*)p;   p += ws_temporal_bytes(total_frames, f);
     ws.first = (int32_t*)p;
-    cudaStream_t stream = (cudaStream_t)cuda_stream;
-    const int omc = dissim_kind == SHARPV_ONE_MINUS_COS;
     if (dtype == SHARPV_F32)
         return launch_score<SHARPV_F32>(tokens, ld_tokens, num_videos, video_frame_offsets, total_frames, f, d,
                                         w, omc, (int)round_mode, min_keep, out_importance, out_spatial,

@@ -1,0 +1,35 @@
+// Interface of the single-kernel implementation of stage one (a) (see score_fused.cu).
+#pragma once
+
+#include "common.cuh"
+
+namespace sharpv {
+
+struct FusedScoreArgs {
+    const void* tokens;
+    sharpv_dtype dtype;
+    int64_t ld_tokens;
+    int num_videos;
+    const int32_t* video_frame_offsets;
+    int F, f, d;
+    float w;
+    int one_minus_cos, round_mode, min_keep;
+    float *out_I, *out_S, *out_T, *out_ratio;
+    int32_t* out_k;
+    void* workspace;            // fused_score_workspace_bytes() bytes, 256-byte aligned
+    int32_t* status_word;       // may be null
+    cudaStream_t stream;
+};
+
+// Shapes the fused kernel covers: rows that split into 256-byte column slices and frames of at
+// most 208 tokens.  Everything else takes the three-kernel path.
+bool fused_score_supported(sharpv_dtype dtype, int f, int d);
+
+// Upper bound over both storage types.
+size_t fused_score_workspace_bytes(int F, int f, int d);
+
+// SHARPV_ERR_UNSUPPORTED means "could not set up (no tensor-map encoder)": nothing was launched
+// and the caller should take the three-kernel path.
+sharpv_status fused_score_launch(const FusedScoreArgs& a);
+
+}  // namespace sharpv

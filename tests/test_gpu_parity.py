@@ -307,6 +307,33 @@ def test_degenerate_inputs():
     assert to_host(gc["mean_cos"])[1] == 0.0
 
 
+@pytest.mark.parametrize("dtype,d", [(W.BF16, 128), (W.F32, 64), (W.BF16, 384), (W.F32, 256)])
+@pytest.mark.parametrize("grid", [1, 3, 14, 15])
+def test_nearly_parallel_rows_and_frame_sizes(dtype, d, grid):
+    """Rows that are almost parallel without being equal (a scaled copy of the previous frame, a frame of
+    identical tokens next to its own rounded mean) in shapes on both sides of the fused kernel's limits
+    (f = 1, 9, 196 inside; f = 225 outside)."""
+    f = grid * grid
+    rng = np.random.default_rng(70 + grid)
+    base = rng.standard_normal((f, d)).astype(np.float32)
+    frames = [base,
+              base * np.float32(1.5),                                   # scaled copy: T ~ 0, not identical
+              np.tile(rng.standard_normal((1, d)).astype(np.float32), (f, 1)),   # uniform frame: S ~ 0
+              base + np.float32(1e-3) * rng.standard_normal((f, d)).astype(np.float32),
+              base.copy()]
+    x = np.concatenate(frames)
+    if dtype == W.BF16:
+        x = W.f32_to_bf16_bits(x)
+    vfo = np.array([0, 3, 5], np.int32)
+    o = orc.score_frames(x, vfo, f, nthreads=NT)
+    g = sv.sharpv_score_frames(to_dev(x), torch.from_numpy(vfo).cuda(), 5, f, want_spatial=True, want_temporal=True)
+    torch.cuda.synchronize()
+    for key in ("spatial", "temporal", "importance", "ratio"):
+        e = rel_err(to_host(g[key]), o[key])
+        assert e <= TIGHT_TOL, f"{key}: rel err {e}"
+    check_budgets(to_host(g["k"]), o, f)
+
+
 def test_run_to_run_bit_reproducible():
     wl, dw = _case("small_ragged")
     F, f = wl.total_frames, wl.f
