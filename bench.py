@@ -46,6 +46,13 @@ def parse_args():
                          "(the paper's reported memory ratio); the paper's default 0.2 keeps all of them")
     ap.add_argument("--w", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stage", default=None, choices=["score", "select", "calibrate", "compact"],
+                    help="profiling aid: after the warm-up run only this entry point --steps times "
+                         "(L2 flushed before each) and print its mean duration")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="override the number of K/V layers (profiling aid: smaller device footprint)")
+    ap.add_argument("--frames", type=int, default=None,
+                    help="override the frame count of a single-video workload (profiling aid)")
     return ap.parse_args()
 
 
@@ -96,8 +103,13 @@ def oracle_step(wl, orc, M, w, nthreads, kv_layers=None):
     return t, idx.size, c["kept_pos"].size
 
 
-def host_workload(name, with_kv_layers=None):
-    wl = W.PRESETS[name]()
+def host_workload(name, with_kv_layers=None, frames=None, layers=None):
+    kw = {}
+    if frames:
+        kw["n_frames"] = frames
+    if layers:
+        kw["num_layers"] = layers
+    wl = W.PRESETS[name](**kw)
     W.fill_tokens(wl)
     W.fill_hidden(wl)
     if with_kv_layers:
@@ -209,7 +221,7 @@ def run_sharpv(args):
     dev = torch.device("cuda", local_rank)
     sv.lib()                                            # fail loudly before any work if not built
 
-    wl = host_workload(args.workload)
+    wl = host_workload(args.workload, frames=args.frames, layers=args.layers)
     F, f, d, T, NV = wl.total_frames, wl.f, wl.d, wl.total_seq_tokens, wl.n_visual
     tdt = torch.float32 if wl.dtype == W.F32 else torch.bfloat16
 
@@ -289,6 +301,23 @@ def run_sharpv(args):
     n_keep = int(o_sel["num_kept"].item())
     t_keep = int(o_cal["kept_seq_offsets"][-1].item())
     assert int(status.item()) == 0, "device status word set"
+
+    if args.stage:
+        fn = dict(stages)[args.stage]
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(args.steps)]
+        for a, b in evs:
+            flush.zero_()
+            a.record(stream)
+            fn()
+            b.record(stream)
+        torch.cuda.synchronize()
+        ms = statistics.fmean(a.elapsed_time(b) for a, b in evs)
+        nbytes = algorithmic_bytes(wl, n_keep, t_keep, args.stage)
+        print(json.dumps({"stage": args.stage, "workload": args.workload, "frames": F, "ms": ms,
+                          "algorithmic_bytes": nbytes, "GBps": nbytes / (ms * 1e-3) / 1e9,
+                          "kept_stage_one": n_keep, "kept_stage_two": t_keep}))
+        return
 
     # The library calls only enqueue kernels (no allocation, no sync), so one step is captured
     # into a CUDA graph and replayed: the GPU never waits for the Python caller.

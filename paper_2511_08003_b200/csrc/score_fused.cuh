@@ -22,7 +22,7 @@ struct FusedScoreArgs {
 };
 
 // Shapes the fused kernel covers: rows that split into 256-byte column slices and frames of at
-// most 208 tokens.  Everything else takes the three-kernel path.
+// most 256 tokens.  Everything else takes the three-kernel path.
 bool fused_score_supported(sharpv_dtype dtype, int f, int d);
 
 // Upper bound over both storage types.

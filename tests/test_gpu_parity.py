@@ -308,11 +308,11 @@ def test_degenerate_inputs():
 
 
 @pytest.mark.parametrize("dtype,d", [(W.BF16, 128), (W.F32, 64), (W.BF16, 384), (W.F32, 256)])
-@pytest.mark.parametrize("grid", [1, 3, 14, 15])
+@pytest.mark.parametrize("grid", [1, 3, 14, 15, 17])
 def test_nearly_parallel_rows_and_frame_sizes(dtype, d, grid):
     """Rows that are almost parallel without being equal (a scaled copy of the previous frame, a frame of
     identical tokens next to its own rounded mean) in shapes on both sides of the fused kernel's limits
-    (f = 1, 9, 196 inside; f = 225 outside)."""
+    (f = 1, 9, 196, 225)."""
     f = grid * grid
     rng = np.random.default_rng(70 + grid)
     base = rng.standard_normal((f, d)).astype(np.float32)
