@@ -4,7 +4,7 @@
 // Kernels:
 //   calibrate_cos_kernel  one warp per packed position: cos(hidden row, visual row), keep flag,
 //                         and an integer count of survivors per chunk of 256 positions
-//   write_kept_kernel     same chunks: chunk base = sum of earlier chunk counts, local scan,
+//   write_kept_kernel     (dependent launch) chunk base = sum of earlier chunk counts, local scan,
 //                         ascending kept positions, per-sequence offsets, capacity check
 //   mean_cos_kernel       (optional) fixed-order mean of the cosines of each sequence
 #include <mutex>
@@ -97,6 +97,7 @@ write_kept_kernel(const uint8_t* __restrict__ flags, const int32_t* __restrict__
     __shared__ int sm[kChunk / 32 + 1];
     __shared__ int s_base;
     const int c = blockIdx.x;
+    cudaGridDependencySynchronize();        // flags and chunk counts come from the kernel in front
     // kept positions before this chunk: fixed-order sum of the earlier chunk counts
     int part = 0;
     for (int i = threadIdx.x; i < c; i += kChunk) part += chunk_counts[i];
@@ -207,8 +208,13 @@ static sharpv_status calibrate_impl(
         calibrate_cos_kernel<SHARPV_BF16><<<ctas, 256, 0, stream>>>(
             (const char*)hidden, ld_hidden * eb, (const char*)visual, ld_visual * eb, nvec, num_seqs, seq_offsets,
             vis_begin, vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, flags, chunk_counts);
-    write_kept_kernel<<<chunks, kChunk, 0, stream>>>(flags, chunk_counts, total_seq_tokens, num_seqs, seq_offsets,
-                                                    capacity, out_kept_pos, out_kept_seq_offsets, status_word);
+    if (cudaGetLastError() != cudaSuccess) return SHARPV_ERR_CUDA;
+    if (launch_dependent(write_kept_kernel, dim3(chunks), dim3(kChunk), 0, stream, (const uint8_t*)flags,
+                         (const int32_t*)chunk_counts, total_seq_tokens, num_seqs, seq_offsets, capacity,
+                         out_kept_pos, out_kept_seq_offsets, status_word) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SHARPV_ERR_CUDA;
+    }
     if (out_mean_cos)
         mean_cos_kernel<<<num_seqs, 256, 0, stream>>>(out_cos, vis_count, vis_offsets, total_visual, out_mean_cos);
     return launch_status();

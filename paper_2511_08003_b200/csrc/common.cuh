@@ -24,6 +24,25 @@ inline sharpv_status launch_status() {
     return cudaGetLastError() == cudaSuccess ? SHARPV_OK : SHARPV_ERR_CUDA;
 }
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while the kernel in
+// front of it on the stream drains, and must call cudaGridDependencySynchronize() before it reads
+// anything that kernel wrote.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                    cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---------------------------------------------------------------------------------------
 // 16-byte vectors of the storage type and their exact fp32 widening
 // ---------------------------------------------------------------------------------------

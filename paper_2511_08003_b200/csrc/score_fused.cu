@@ -25,13 +25,12 @@ namespace {
 
 constexpr int kSliceBytes = 256;
 constexpr int kThreads = 512;           // 16 warps; a warp = 4 row groups x 8 lanes (two vectors per lane)
-constexpr int kWarps = kThreads / 32;
 constexpr int kRowGroups = kThreads / 8;
 constexpr int kRows = 4;                // row slots per thread: frames of up to 256 tokens
 constexpr int kMaxTokensFused = 256;
 constexpr int kSmemBudget = 227 * 1024;
 constexpr uint32_t kSpinLimit = 1u << 22;      // polls of one mbarrier before a wait gives up
-constexpr int kFinThreads = 256;
+constexpr int kFinThreads = 1024;
 
 struct FusedParams {
     const char* tokens;
@@ -77,6 +76,50 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
         ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
 
+// Two fp32 values in one 64-bit register, the operand form of the packed fp32 instructions.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pk(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ float hsum(f32x2 v) {
+    float lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+    return lo + hi;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// one 32-bit word of two bf16 -> the two exact fp32 values (a bf16 is the upper half of an fp32):
+// two byte permutes written straight into the halves of the 64-bit result
+__device__ __forceinline__ f32x2 widen_bf16x2(uint32_t w) {
+    f32x2 r;
+    asm("{\n\t.reg .b32 lo, hi;\n\t"
+        "prmt.b32 lo, %1, %2, 0x1044;\n\t"
+        "prmt.b32 hi, %1, %2, 0x3244;\n\t"
+        "mov.b64 %0, {lo, hi};\n\t}"
+        : "=l"(r) : "r"(w), "r"(0u));
+    return r;
+}
+__device__ __forceinline__ f32x2 pair_f32(uint32_t lo, uint32_t hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+
 // 8 lanes x 16 values (x[4*slot + j], 4 slots) -> lane L of the group ends with x[0], x[1] =
 // values 2*(L&1), 2*(L&1)+1 of slot L>>1.  Fixed pairing, hence a fixed summation order.
 __device__ __forceinline__ void group8_reduce_scatter(float (&x)[16], int lane8) {
@@ -115,7 +158,7 @@ template <int DT>
 struct Pass {
     using E = Elem<DT>;
     static constexpr int P = E::kPerVec;                    // elements per 16-byte vector
-    static constexpr int H = P / 2;                         // float2 pairs per vector
+    static constexpr int H = P / 2;                         // packed pairs per vector
     static constexpr int SE = kSliceBytes / E::kBytes;      // elements per slice row
 
     const CUtensorMap* tmap;
@@ -126,60 +169,67 @@ struct Pass {
     float* mean_s;          // [SE]
     uint64_t* bars;         // [nbuf]
     volatile int* abort_flag;
-    int64_t u0;
     int Q, halo;
+    int load_s, load_t;     // (slice, frame) of the next tile to request (thread 0 only)
 
     // per-thread state carried from frame to frame
     uint4 prev[kRows][2];   // previous frame's rows of this thread (two vectors each)
-    float2 mprev[2][H];     // previous frame's mean over this thread's columns
+    f32x2 mprev[2][H];      // previous frame's mean over this thread's columns
     float bb[kRows];        // this thread's share of ||previous row||^2
 
-    int warp, g, j, rgid;
+    int tid, warp, g, j, rgid;
 
-    __device__ __forceinline__ int row_of(int r) const { return warp + kWarps * (4 * r + g); }
-
-    __device__ __forceinline__ void issue_load(int q) const {
+    // requests tile q; tiles are requested in unit order, so (load_s, load_t) just advances
+    __device__ __forceinline__ void issue_load(int q) {
         const FusedParams& pp = *p;
-        const int64_t u = u0 + q - halo;
-        int t, s;
-        if (halo && q == 0) { s = (int)(u0 / pp.F); t = (int)(u0 % pp.F) - 1; }
-        else { s = (int)(u / pp.F); t = (int)(u % pp.F); }
-        uint64_t* bar = bars + (q % pp.nbuf);
+        const int slot = q % pp.nbuf;
+        uint64_t* bar = bars + slot;
         mbar_expect_tx(bar, pp.tile_bytes);
-        tma_load_2d(tiles + (size_t)(q % pp.nbuf) * pp.tile_stride, tmap, s * kSliceBytes, t * pp.f, bar);
+        tma_load_2d(tiles + (size_t)slot * pp.tile_stride, tmap, load_s * kSliceBytes, load_t * pp.f, bar);
+        if (++load_t == pp.F) { load_t = 0; ++load_s; }
     }
 
-    __device__ __forceinline__ const unsigned char* wait_tile(int q) const {
-        const int nb = p->nbuf;
-        if (!mbar_wait(bars + (q % nb), (uint32_t)((q / nb) & 1))) *abort_flag = 1;
-        return tiles + (size_t)(q % nb) * p->tile_stride;
+    __device__ __forceinline__ const unsigned char* wait_tile(int slot, uint32_t phase) const {
+        if (!mbar_wait(bars + slot, phase)) *abort_flag = 1;
+        return tiles + (size_t)slot * p->tile_stride;
     }
 
-    __device__ __forceinline__ static void to_pairs(const uint4& v, float2 (&o)[H]) {
-        float x[P];
-        E::widen(v, x);
-#pragma unroll
-        for (int i = 0; i < H; ++i) o[i] = make_float2(x[2 * i], x[2 * i + 1]);
+    __device__ __forceinline__ static void to_pairs(const uint4& v, f32x2 (&o)[H]) {
+        if (DT == SHARPV_BF16) {
+            o[0] = widen_bf16x2(v.x); o[1] = widen_bf16x2(v.y);
+            o[H - 2] = widen_bf16x2(v.z); o[H - 1] = widen_bf16x2(v.w);
+        } else {
+            o[0] = pair_f32(v.x, v.y); o[H - 1] = pair_f32(v.z, v.w);
+        }
+    }
+
+    // Row slot r of this thread is row 64 r + 4 warp + g (g = lane group): a warp owns four
+    // consecutive rows per slot.  A slot is visited when its first row exists (a warp-uniform test);
+    // lane groups whose row lies beyond the frame read the zero rows that pad every tile buffer to a
+    // multiple of four rows, so no lane ever branches on its own row.
+    __device__ __forceinline__ bool slot_live(int r) const { return 64 * r + 4 * warp < p->f; }
+    __device__ __forceinline__ int slot_row(int r) const { return 64 * r + 4 * warp + g; }
+    __device__ __forceinline__ const unsigned char* my_rows(const unsigned char* tile) const {
+        return tile + (4 * warp + g) * kSliceBytes + j * 16;
     }
 
     // Frame in front of the first unit: registers only.
-    __device__ __forceinline__ void load_halo(int q) {
-        const unsigned char* tile = wait_tile(q);
+    __device__ __forceinline__ void load_halo(const unsigned char* tile) {
+        const unsigned char* base = my_rows(tile);
 #pragma unroll
         for (int r = 0; r < kRows; ++r) {
-            const int row = row_of(r);
-            float2 acc = make_float2(0.f, 0.f);
-            if (row < p->f) {
+            f32x2 acc = pk(0.f, 0.f);
+            if (slot_live(r)) {
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    prev[r][h] = *reinterpret_cast<const uint4*>(tile + row * kSliceBytes + (j + 8 * h) * 16);
-                    float2 b2[H];
+                    prev[r][h] = *reinterpret_cast<const uint4*>(base + r * (64 * kSliceBytes) + h * 128);
+                    f32x2 b2[H];
                     to_pairs(prev[r][h], b2);
 #pragma unroll
-                    for (int i = 0; i < H; ++i) acc = __ffma2_rn(b2[i], b2[i], acc);
+                    for (int i = 0; i < H; ++i) acc = fma2(b2[i], b2[i], acc);
                 }
             }
-            bb[r] = acc.x + acc.y;
+            bb[r] = hsum(acc);
         }
     }
 
@@ -191,95 +241,107 @@ struct Pass {
         for (int i = 0; i < 16; ++i) x[i] = 0.f;
 #pragma unroll
         for (int r = 0; r < kRows; ++r) {
-            if (row_of(r) < p->f) {
-                float2 acc = make_float2(0.f, 0.f);
+            if (slot_live(r)) {
+                f32x2 acc = pk(0.f, 0.f);
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    float2 b2[H];
+                    f32x2 b2[H];
                     to_pairs(prev[r][h], b2);
 #pragma unroll
-                    for (int i = 0; i < H; ++i) acc = __ffma2_rn(b2[i], mprev[h][i], acc);
+                    for (int i = 0; i < H; ++i) acc = fma2(b2[i], mprev[h][i], acc);
                 }
-                x[4 * r + 3] = acc.x + acc.y;
+                x[4 * r + 3] = hsum(acc);
             }
         }
         group8_reduce_scatter(x, j);
-        const int row = warp + kWarps * (4 * (j >> 1) + g);
+        const int row = slot_row(j >> 1);
         if ((j & 1) && row < p->f) p->part[((int64_t)t_prev * p->nsl + s) * p->f + row].w = x[1];
     }
 
-    // One unit: tile q = (slice s, frame t).
-    //   has_prev  the registers hold frame t-1 of this slice
-    //   own_prev  ... and it was a unit of this CTA, so its <row, mean> is computed here
-    // Returns false when the CTA must stop (a bounded wait ran out).
-    __device__ __forceinline__ bool unit(int q, int s, int t, bool has_prev, bool own_prev) {
-        const FusedParams& pp = *p;
-        const bool temporal = has_prev && !frame_is_first(pp.video_frame_offsets, pp.num_videos, t);
-        const unsigned char* tile = wait_tile(q);
+    // Slots [R0, R1) of one tile, without a branch: everything the frame contributes per row.
+    //   HAS_PREV  the registers hold frame t-1 of this slice
+    //   TEMPORAL  ... and frame t continues the same video, so ||a-b||^2 is wanted
+    //   OWN_PREV  ... and frame t-1 was a unit of this CTA, so its <row, mean> is computed here
+    template <int R0, int R1, bool HAS_PREV, bool TEMPORAL, bool OWN_PREV>
+    __device__ __forceinline__ void slots(const unsigned char* base, f32x2 (&colsum)[2][H], float (&x)[16]) {
+        uint4 a4[R1 - R0][2];
+#pragma unroll
+        for (int r = R0; r < R1; ++r)
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+                a4[r - R0][h] = *reinterpret_cast<const uint4*>(base + r * (64 * kSliceBytes) + h * 128);
+#pragma unroll
+        for (int r = R0; r < R1; ++r) {
+            f32x2 aa = pk(0.f, 0.f), db = aa, bm = aa;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                f32x2 a2[H];
+                to_pairs(a4[r - R0][h], a2);
+#pragma unroll
+                for (int i = 0; i < H; ++i) {
+                    colsum[h][i] = add2(colsum[h][i], a2[i]);
+                    aa = fma2(a2[i], a2[i], aa);
+                }
+                if (HAS_PREV && (TEMPORAL || OWN_PREV)) {
+                    f32x2 b2[H];
+                    to_pairs(prev[r][h], b2);
+#pragma unroll
+                    for (int i = 0; i < H; ++i) {
+                        if (TEMPORAL) {
+                            const f32x2 e = sub2(a2[i], b2[i]);
+                            db = fma2(e, e, db);
+                        }
+                        if (OWN_PREV) bm = fma2(b2[i], mprev[h][i], bm);
+                    }
+                }
+                prev[r][h] = a4[r - R0][h];
+            }
+            x[4 * r + 0] = hsum(aa);
+            x[4 * r + 1] = hsum(db);
+            x[4 * r + 2] = HAS_PREV ? bb[r] : 0.f;
+            x[4 * r + 3] = hsum(bm);
+            bb[r] = x[4 * r + 0];
+        }
+    }
 
-        float2 colsum[2][H];
+    // One unit: the tile of (slice s, frame t) in buffer `slot`; q is its place in the load order.
+    // Returns false when the CTA must stop (a bounded wait ran out).
+    template <bool HAS_PREV, bool TEMPORAL, bool OWN_PREV>
+    __device__ __forceinline__ bool unit(int q, int slot, uint32_t phase, int s, int t) {
+        const FusedParams& pp = *p;
+        const unsigned char* base = my_rows(wait_tile(slot, phase));
+
+        f32x2 colsum[2][H];
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
-            for (int i = 0; i < H; ++i) colsum[h][i] = make_float2(0.f, 0.f);
+            for (int i = 0; i < H; ++i) colsum[h][i] = pk(0.f, 0.f);
         float x[16];
-        const float2 one = make_float2(1.f, 1.f), neg1 = make_float2(-1.f, -1.f);
 #pragma unroll
-        for (int r = 0; r < kRows; ++r) {
-            const int row = row_of(r);
-            float2 aa = make_float2(0.f, 0.f), db = aa, bm = aa;
-            if (row < pp.f) {
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint4 a4 = *reinterpret_cast<const uint4*>(tile + row * kSliceBytes + (j + 8 * h) * 16);
-                    float2 a2[H];
-                    to_pairs(a4, a2);
-#pragma unroll
-                    for (int i = 0; i < H; ++i) {
-                        colsum[h][i] = __ffma2_rn(a2[i], one, colsum[h][i]);
-                        aa = __ffma2_rn(a2[i], a2[i], aa);
-                    }
-                    if (has_prev) {
-                        float2 b2[H];
-                        to_pairs(prev[r][h], b2);
-                        if (temporal) {
-#pragma unroll
-                            for (int i = 0; i < H; ++i) {
-                                const float2 e = __ffma2_rn(b2[i], neg1, a2[i]);        // a - b
-                                db = __ffma2_rn(e, e, db);
-                            }
-                        }
-                        if (own_prev) {
-#pragma unroll
-                            for (int i = 0; i < H; ++i) bm = __ffma2_rn(b2[i], mprev[h][i], bm);
-                        }
-                    }
-                    prev[r][h] = a4;
-                }
-            }
-            x[4 * r + 0] = aa.x + aa.y;
-            x[4 * r + 1] = db.x + db.y;
-            x[4 * r + 2] = has_prev ? bb[r] : 0.f;
-            x[4 * r + 3] = bm.x + bm.y;
-            bb[r] = x[4 * r + 0];
+        for (int i = 0; i < 16; ++i) x[i] = 0.f;
+        if (slot_live(2)) {                     // the usual case: a straight run over three slots
+            slots<0, 2, HAS_PREV, TEMPORAL, OWN_PREV>(base, colsum, x);
+            slots<2, 3, HAS_PREV, TEMPORAL, OWN_PREV>(base, colsum, x);
+            if (slot_live(3)) slots<3, 4, HAS_PREV, TEMPORAL, OWN_PREV>(base, colsum, x);
+        } else {
+            if (slot_live(0)) slots<0, 1, HAS_PREV, TEMPORAL, OWN_PREV>(base, colsum, x);
+            if (slot_live(1)) slots<1, 2, HAS_PREV, TEMPORAL, OWN_PREV>(base, colsum, x);
         }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             float* dst = cs + rgid * SE + (j + 8 * h) * P;
 #pragma unroll
             for (int i = 0; i < H; i += 2)
-                *reinterpret_cast<float4*>(dst + 2 * i) =
-                    make_float4(colsum[h][i].x, colsum[h][i].y, colsum[h][i + 1].x, colsum[h][i + 1].y);
+                *reinterpret_cast<ulonglong2*>(dst + 2 * i) = make_ulonglong2(colsum[h][i], colsum[h][i + 1]);
         }
         __syncthreads();                            // tile buffer free, column partials visible
         if (*abort_flag) return false;
-        const int tid = threadIdx.x;
         if (tid == 0 && q + pp.nbuf < Q) issue_load(q + pp.nbuf);
         // column sums over the 64 row groups: fixed order, two levels
         for (int e = tid; e < 4 * SE; e += kThreads) {
             const int col = e % SE, quarter = e / SE;
             float sum = 0.f;
-#pragma unroll 8
+#pragma unroll
             for (int i = 0; i < kRowGroups / 4; ++i) sum += cs[(quarter * (kRowGroups / 4) + i) * SE + col];
             cs2[quarter * SE + col] = sum;
         }
@@ -287,12 +349,12 @@ struct Pass {
         // per-row partial sums of the slice (overlaps the mean reduction of the other warps)
         group8_reduce_scatter(x, j);
         {
-            const int row = warp + kWarps * (4 * (j >> 1) + g);
+            const int row = slot_row(j >> 1);
             if (row < pp.f) {
                 float4* rec = pp.part + ((int64_t)t * pp.nsl + s) * pp.f + row;
                 if (j & 1) {
                     rec->z = x[0];                                              // ||b||^2
-                    if (own_prev) pp.part[((int64_t)(t - 1) * pp.nsl + s) * pp.f + row].w = x[1];
+                    if (OWN_PREV) (rec - (int64_t)pp.nsl * pp.f)->w = x[1];     // frame t-1: <b, mean>
                 } else {
                     *reinterpret_cast<float2*>(rec) = make_float2(x[0], x[1]);  // ||a||^2, ||a-b||^2
                 }
@@ -309,8 +371,18 @@ struct Pass {
         for (int h = 0; h < 2; ++h)
 #pragma unroll
             for (int i = 0; i < H; ++i)
-                mprev[h][i] = *reinterpret_cast<const float2*>(mean_s + (j + 8 * h) * P + 2 * i);
+                mprev[h][i] = *reinterpret_cast<const f32x2*>(mean_s + (j + 8 * h) * P + 2 * i);
         return true;
+    }
+
+    __device__ __forceinline__ bool unit_dispatch(int q, int slot, uint32_t phase, int s, int t, bool has_prev,
+                                                  bool own_prev, bool is_first) {
+        if (!has_prev) return unit<false, false, false>(q, slot, phase, s, t);
+        if (!is_first)
+            return own_prev ? unit<true, true, true>(q, slot, phase, s, t)
+                            : unit<true, true, false>(q, slot, phase, s, t);
+        return own_prev ? unit<true, false, true>(q, slot, phase, s, t)
+                        : unit<true, false, false>(q, slot, phase, s, t);
     }
 };
 
@@ -329,16 +401,26 @@ score_pass_kernel(const __grid_constant__ CUtensorMap tmap, const FusedParams p,
     c.bars = reinterpret_cast<uint64_t*>(c.mean_s + SE);
     c.abort_flag = reinterpret_cast<volatile int*>(c.bars + 4);
 
-    const int64_t U = (int64_t)p.nsl * p.F;
-    c.u0 = U * blockIdx.x / gridDim.x;
-    const int64_t u1 = U * (blockIdx.x + 1) / gridDim.x;
     // let the finaliser's CTAs be scheduled as soon as SMs free up; they wait for this whole grid
     cudaTriggerProgrammaticLaunchCompletion();
-    if (c.u0 >= u1) return;
-    c.halo = frame_is_first(p.video_frame_offsets, p.num_videos, (int)(c.u0 % p.F)) ? 0 : 1;
-    c.Q = (int)(u1 - c.u0) + c.halo;
+    const int64_t U = (int64_t)p.nsl * p.F;
+    const int64_t u0 = U * blockIdx.x / gridDim.x;
+    const int64_t u1 = U * (blockIdx.x + 1) / gridDim.x;
+    if (u0 >= u1) return;
+    int s = (int)(u0 / p.F), t = (int)(u0 % p.F);
+
+    // videos: `vid` is the video of frame t, `next_start` the first frame of the next one
+    int vid = upper_segment(p.video_frame_offsets, p.num_videos, t);
+    bool is_first = __ldg(p.video_frame_offsets + vid) == t;
+    int next_start = __ldg(p.video_frame_offsets + vid + 1);
+
+    c.halo = is_first ? 0 : 1;
+    c.Q = (int)(u1 - u0) + c.halo;
+    c.load_s = s;
+    c.load_t = t - c.halo;
 
     const int tid = threadIdx.x, lane = tid & 31;
+    c.tid = tid;
     c.warp = tid >> 5;
     c.g = lane >> 3;
     c.j = lane & 7;
@@ -348,6 +430,12 @@ score_pass_kernel(const __grid_constant__ CUtensorMap tmap, const FusedParams p,
         *c.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    // rows beyond the frame in every tile buffer stay zero for the whole kernel (TMA writes f rows)
+    for (int b = 0; b < p.nbuf; ++b) {
+        uint4* pad = reinterpret_cast<uint4*>(c.tiles + (size_t)b * p.tile_stride + p.tile_bytes);
+        const int n = (int)((p.tile_stride - p.tile_bytes) / 16);
+        for (int i = tid; i < n; i += kThreads) pad[i] = make_uint4(0u, 0u, 0u, 0u);
     }
     __syncthreads();
     if (tid == 0)
@@ -360,31 +448,46 @@ score_pass_kernel(const __grid_constant__ CUtensorMap tmap, const FusedParams p,
         c.bb[r] = 0.f;
     }
 
-    int q = 0;
+    int q = 0, slot = 0;
+    uint32_t phase = 0;
     bool ok = true, has_prev = false, own_prev = false;
     if (c.halo) {
-        c.load_halo(0);
+        c.load_halo(c.wait_tile(0, 0));
         __syncthreads();
         ok = *c.abort_flag == 0;
         if (ok && tid == 0 && p.nbuf < c.Q) c.issue_load(p.nbuf);
         q = 1;
+        if (++slot == p.nbuf) { slot = 0; phase ^= 1; }
         has_prev = true;
     }
-    int s_cur = (int)(c.u0 / p.F);
-    for (int64_t u = c.u0; ok && u < u1; ++u, ++q) {
-        const int s = (int)(u / p.F), t = (int)(u % p.F);
-        if (s != s_cur) {                           // the range crosses into the next slice
-            if (own_prev) c.flush_prev(s_cur, p.F - 1);
-            has_prev = false;
-            own_prev = false;
-            s_cur = s;
-        }
-        ok = c.unit(q, s, t, has_prev, own_prev);
+    const int n_units = (int)(u1 - u0);
+    for (int i = 0; ok && i < n_units; ++i) {
+        ok = c.unit_dispatch(q, slot, phase, s, t, has_prev, own_prev, is_first);
         has_prev = true;
         own_prev = true;
+        ++q;
+        if (++slot == p.nbuf) { slot = 0; phase ^= 1; }
+        // next unit
+        if (++t == p.F) {                           // the range crosses into the next slice
+            if (ok) c.flush_prev(s, p.F - 1);
+            t = 0;
+            ++s;
+            has_prev = false;
+            own_prev = false;
+            vid = upper_segment(p.video_frame_offsets, p.num_videos, 0);
+            next_start = __ldg(p.video_frame_offsets + vid + 1);
+            is_first = true;
+        } else {
+            is_first = false;
+            while (t >= next_start && vid + 1 < p.num_videos) {     // skips videos without frames
+                ++vid;
+                is_first = true;
+                next_start = __ldg(p.video_frame_offsets + vid + 1);
+            }
+        }
     }
     if (ok) {
-        if (own_prev) c.flush_prev(s_cur, (int)((u1 - 1) % p.F));
+        if (own_prev) c.flush_prev((int)((u1 - 1) / p.F), (int)((u1 - 1) % p.F));
     } else {
         // A wait on the CTA's own loads ran out.  Report it, then give the loads that are still in
         // flight one more bounded wait each, so that nothing lands in shared memory after exit.
@@ -405,48 +508,55 @@ __device__ __forceinline__ float dissim_sq_from_dot(float saa, float sbb, float 
 }
 
 // One CTA per frame: adds the slices in a fixed order, writes S, T, I, ratio_t and k_t.
+// 1024 threads = 4 groups x 256 rows; group q adds slices q, q+4, ... (all loads in flight at once),
+// then the four group sums are added in order.
 template <int DT>
 __global__ void __launch_bounds__(kFinThreads)
 score_finalize_kernel(const FusedParams p) {
+    __shared__ float4 g_sum[4][kMaxTokensFused];
     __shared__ float f_s2[kMaxTokensFused], f_t2[kMaxTokensFused], f_aa[kMaxTokensFused], f_bb[kMaxTokensFused];
     __shared__ int f_fl[kMaxTokensFused];
     __shared__ float red[kFinThreads / 32];
     const int t = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int row = tid & (kMaxTokensFused - 1), grp = tid >> 8;
     const bool is_first = frame_is_first(p.video_frame_offsets, p.num_videos, t);
     // everything the pass kernel wrote is visible after this point
     cudaGridDependencySynchronize();
 
-    // ||mean||^2, fixed order
+    // every load of this thread is issued before the first one is used: one memory round trip
     const float* mean = p.mean + (int64_t)t * p.d;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float sm = 0.f;
-    for (int c = tid * 4; c < p.d; c += kFinThreads * 4) {
-        const float4 m = __ldcg(reinterpret_cast<const float4*>(mean + c));
-        sm = fmaf(m.x, m.x, sm); sm = fmaf(m.y, m.y, sm); sm = fmaf(m.z, m.z, sm); sm = fmaf(m.w, m.w, sm);
+    const float4* src = p.part + ((int64_t)t * p.nsl) * p.f + row;
+    for (int s0 = grp; s0 < p.nsl; s0 += 32) {
+        float4 q[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int s = s0 + 4 * i;
+            q[i] = (row < p.f && s < p.nsl) ? __ldcg(src + (int64_t)s * p.f) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (s0 == grp) {
+            for (int c = tid * 4; c < p.d; c += kFinThreads * 4) {
+                const float4 m = __ldcg(reinterpret_cast<const float4*>(mean + c));
+                sm = fmaf(m.x, m.x, sm); sm = fmaf(m.y, m.y, sm); sm = fmaf(m.z, m.z, sm); sm = fmaf(m.w, m.w, sm);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { acc.x += q[i].x; acc.y += q[i].y; acc.z += q[i].z; acc.w += q[i].w; }
     }
+    g_sum[grp][row] = acc;
     sm = warp_sum(sm);
     if (lane == 0) red[warp] = sm;
     __syncthreads();
     float smm = 0.f;
 #pragma unroll
     for (int i = 0; i < kFinThreads / 32; ++i) smm += red[i];
-    __syncthreads();
 
     if (tid < p.f) {
-        float aa = 0.f, db = 0.f, bb = 0.f, am = 0.f;
-        const float4* src = p.part + ((int64_t)t * p.nsl) * p.f + tid;
-        int s = 0;
-        for (; s + 4 <= p.nsl; s += 4) {
-            float4 q[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) q[i] = __ldcg(src + (int64_t)(s + i) * p.f);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { aa += q[i].x; db += q[i].y; bb += q[i].z; am += q[i].w; }
-        }
-        for (; s < p.nsl; ++s) {
-            const float4 q = __ldcg(src + (int64_t)s * p.f);
-            aa += q.x; db += q.y; bb += q.z; am += q.w;
-        }
+        const float4 a0 = g_sum[0][tid], a1 = g_sum[1][tid], a2 = g_sum[2][tid], a3 = g_sum[3][tid];
+        const float aa = (a0.x + a1.x) + (a2.x + a3.x), db = (a0.y + a1.y) + (a2.y + a3.y);
+        const float bb = (a0.z + a1.z) + (a2.z + a3.z), am = (a0.w + a1.w) + (a2.w + a3.w);
         const float s2 = dissim_sq_from_dot(aa, smm, am);
         const float t2 = is_first ? 0.f : dissim_sq_from_sums(aa, bb, db);
         int fl = 0;
@@ -456,19 +566,19 @@ score_finalize_kernel(const FusedParams p) {
     }
     __syncthreads();
     // nearly parallel rows: exact re-evaluation from the rows themselves (rare)
-    for (int row = warp; row < p.f; row += kFinThreads / 32) {
-        const int fl = f_fl[row];
+    for (int r = warp; r < p.f; r += kFinThreads / 32) {
+        const int fl = f_fl[r];
         if (fl) {
-            const char* pa = p.tokens + ((int64_t)t * p.f + row) * p.row_bytes_ld;
+            const char* pa = p.tokens + ((int64_t)t * p.f + r) * p.row_bytes_ld;
             const char* pb = pa - (int64_t)p.f * p.row_bytes_ld;
-            const float ia = 1.f / fmaxf(sqrtf(f_aa[row]), kNormEps);
-            const float ib = 1.f / fmaxf(sqrtf(f_bb[row]), kNormEps);
+            const float ia = 1.f / fmaxf(sqrtf(f_aa[r]), kNormEps);
+            const float ib = 1.f / fmaxf(sqrtf(f_bb[r]), kNormEps);
             const float im = 1.f / fmaxf(sqrtf(smm), kNormEps);
             float es, et;
             refine_row<DT>(pa, pb, mean, p.nvec, lane, (fl & 1) != 0, (fl & 2) != 0, ia, ib, im, es, et);
             if (lane == 0) {
-                if (fl & 1) f_s2[row] = es;
-                if (fl & 2) f_t2[row] = et;
+                if (fl & 1) f_s2[r] = es;
+                if (fl & 2) f_t2[r] = et;
             }
         }
     }
@@ -484,7 +594,7 @@ score_finalize_kernel(const FusedParams p) {
         tsq = T * T;
     }
     tsq = warp_sum(tsq);
-    if (lane == 0) red[warp] = tsq;
+    if (lane == 0) red[warp] = tsq;         // rows live in the first 8 warps; the others add zeros
     __syncthreads();
     if (tid == 0) {
         float tot = 0.f;
@@ -534,17 +644,8 @@ sharpv_status launch(const FusedScoreArgs& a, const CUtensorMap& tmap, FusedPara
     if (cudaGetLastError() != cudaSuccess) return SHARPV_ERR_CUDA;
 
     // the finaliser starts while the pass drains and waits for it with cudaGridDependencySynchronize
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)a.F);
-    cfg.blockDim = dim3(kFinThreads);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = a.stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, score_finalize_kernel<DT>, p) != cudaSuccess) {
+    if (launch_dependent(score_finalize_kernel<DT>, dim3((unsigned)a.F), dim3(kFinThreads), 0, a.stream, p) !=
+        cudaSuccess) {
         (void)cudaGetLastError();
         return SHARPV_ERR_CUDA;
     }
@@ -582,7 +683,7 @@ sharpv_status fused_score_launch(const FusedScoreArgs& a) {
     p.mean = (float*)w;       w += align_up((size_t)a.F * a.d * 4, 256);
     p.part = (float4*)w;
     p.tile_bytes = (uint32_t)a.f * kSliceBytes;
-    p.tile_stride = (uint32_t)align_up((size_t)p.tile_bytes, 128);
+    p.tile_stride = (uint32_t)((a.f + 3) / 4 * 4) * kSliceBytes;   // whole groups of four rows; the tail stays zero
 
     // the token matrix as a byte tensor [rows, d * elem_bytes]; one box is one (frame, slice) tile
     CUtensorMap tmap;

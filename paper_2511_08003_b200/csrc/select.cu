@@ -4,10 +4,11 @@
 //
 // Kernels:
 //   count_above_kernel   (threshold variant only) per-frame count of I > K
-//   scan_budgets_kernel  one CTA: exclusive scan of the clamped budgets -> kept_offsets
-//   select_frame_kernel  one CTA per frame: radix select of the k-th largest key in shared
-//                        memory, then an index-ordered scan that writes ascending indices
-//   gather_rows_kernel   one warp per kept row, 128-bit copies
+//   select_frame_kernel  one CTA per frame: its offset (sum of the budgets in front of it), a radix
+//                        select of the k-th largest key in shared memory, then an index-ordered
+//                        scan that writes ascending indices
+//   gather_rows_kernel   one warp per kept row, 128-bit copies; launched as a dependent of the
+//                        selection so that its start-up overlaps it
 #include "common.cuh"
 
 namespace sharpv {
@@ -38,33 +39,11 @@ count_above_kernel(const float* __restrict__ importance, float K, int f, int32_t
     }
 }
 
-__global__ void __launch_bounds__(1024)
-scan_budgets_kernel(const int32_t* __restrict__ k, int F, int f, int64_t capacity,
-                    int32_t* __restrict__ kept_offsets, int32_t* __restrict__ num_kept,
-                    int32_t* status_word) {
-    __shared__ int sm[1024 / 32 + 1];
-    int carry = 0;
-    for (int base = 0; base < F; base += 1024) {
-        const int t = base + threadIdx.x;
-        int v = 0;
-        if (t < F) v = min(max(k[t], 0), f);
-        int total;
-        const int ex = block_exclusive_scan<1024>(v, sm, total);
-        if (t < F) kept_offsets[t] = carry + ex;
-        carry += total;
-    }
-    if (threadIdx.x == 0) {
-        kept_offsets[F] = carry;
-        if (num_kept) *num_kept = carry;
-        if ((int64_t)carry > capacity) report(status_word, SHARPV_ERR_CAPACITY);
-    }
-}
-
 // mode 0: top-k with budgets k[t];  mode 1: keep I > K
 __global__ void __launch_bounds__(kSelectThreads)
-select_frame_kernel(const float* __restrict__ importance, const int32_t* __restrict__ k,
-                    const int32_t* __restrict__ kept_offsets, int f, int64_t capacity, int mode, float K,
-                    int32_t* __restrict__ out_kept_index) {
+select_frame_kernel(const float* __restrict__ importance, const int32_t* __restrict__ k, int F, int f,
+                    int64_t capacity, int mode, float K, int32_t* __restrict__ kept_offsets,
+                    int32_t* __restrict__ num_kept, int32_t* __restrict__ out_kept_index, int32_t* status_word) {
     extern __shared__ uint32_t keys[];                 // [f]
     __shared__ int hist[256];
     __shared__ int scan_sm[kSelectThreads / 32 + 1];
@@ -72,8 +51,23 @@ select_frame_kernel(const float* __restrict__ importance, const int32_t* __restr
 
     const int t = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t out_base = kept_offsets[t];
     const float* imp = importance + (int64_t)t * f;
+
+    // exclusive scan of the (clamped) budgets: every CTA adds up the frames in front of it
+    int part = 0;
+    for (int i = tid; i < t; i += kSelectThreads) part += min(max(k[i], 0), f);
+    int before;
+    block_exclusive_scan<kSelectThreads>(part, scan_sm, before);
+    const int64_t out_base = before;
+    if (tid == 0) {
+        kept_offsets[t] = before;
+        if (t == F - 1) {
+            const int total = before + min(max(k[t], 0), f);
+            kept_offsets[F] = total;
+            if (num_kept) *num_kept = total;
+            if ((int64_t)total > capacity) report(status_word, SHARPV_ERR_CAPACITY);
+        }
+    }
 
     uint32_t kth = 0;
     int remaining = 0;
@@ -167,6 +161,7 @@ __global__ void __launch_bounds__(256)
 gather_rows_kernel(const char* __restrict__ src, int64_t src_row_bytes, int nvec,
                    const int32_t* __restrict__ index, const int32_t* __restrict__ count_ptr,
                    int64_t capacity, char* __restrict__ dst, int64_t dst_row_bytes) {
+    cudaGridDependencySynchronize();        // the index list comes from the kernel in front
     const int lane = threadIdx.x & 31;
     const int64_t j = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int64_t n = min((int64_t)__ldg(count_ptr), capacity);
@@ -216,20 +211,27 @@ sharpv_status select_impl(int mode, const float* importance, const int32_t* k, f
         count_above_kernel<<<F, kSelectThreads, 0, stream>>>(importance, K, f, counts);
         budgets = counts;
     }
-    scan_budgets_kernel<<<1, 1024, 0, stream>>>(budgets, F, f, capacity, out_kept_offsets, out_num_kept,
-                                                status_word);
-    if (F > 0) {
-        select_frame_kernel<<<F, kSelectThreads, (size_t)f * 4, stream>>>(
-            importance, budgets, out_kept_offsets, f, capacity, mode, K, out_kept_index);
-        if (out_tokens && capacity > 0) {
-            const int64_t rows = capacity < (int64_t)F * f ? capacity : (int64_t)F * f;
-            const int nvec = d * eb / 16;
-            gather_rows_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, stream>>>(
-                (const char*)tokens, ld_tokens * eb, nvec, out_kept_index, out_kept_offsets + F, capacity,
-                (char*)out_tokens, (int64_t)d * eb);
+    if (F == 0) {
+        if (cudaMemsetAsync(out_kept_offsets, 0, sizeof(int32_t), stream) != cudaSuccess) return SHARPV_ERR_CUDA;
+        if (out_num_kept && cudaMemsetAsync(out_num_kept, 0, sizeof(int32_t), stream) != cudaSuccess)
+            return SHARPV_ERR_CUDA;
+        return SHARPV_OK;
+    }
+    select_frame_kernel<<<F, kSelectThreads, (size_t)f * 4, stream>>>(
+        importance, budgets, F, f, capacity, mode, K, out_kept_offsets, out_num_kept, out_kept_index, status_word);
+    if (cudaGetLastError() != cudaSuccess) return SHARPV_ERR_CUDA;
+    if (out_tokens && capacity > 0) {
+        const int64_t rows = capacity < (int64_t)F * f ? capacity : (int64_t)F * f;
+        const int nvec = d * eb / 16;
+        if (launch_dependent(gather_rows_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, stream,
+                             (const char*)tokens, ld_tokens * eb, nvec, (const int32_t*)out_kept_index,
+                             (const int32_t*)(out_kept_offsets + F), capacity, (char*)out_tokens,
+                             (int64_t)d * eb) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return SHARPV_ERR_CUDA;
         }
     }
-    return launch_status();
+    return SHARPV_OK;
 }
 
 }  // namespace
