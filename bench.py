@@ -29,9 +29,9 @@ METRIC = "pruning throughput (visual tokens/s)"
 UNIT = "visual tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # kernels launched per step by each entry point (score, select, calibrate, compact)
-LAUNCHES_PER_STEP = {"score": 3, "select": 3, "calibrate": 2, "compact": 1}
+LAUNCHES_PER_STEP = {"score": 2, "select": 2, "calibrate": 2, "compact": 1}
 # DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/); None = not captured
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {("onevision_7b", "compact"): 267_609_600}   # profiles/kv_compact_kernel_onevision_7b.md
 
 
 def parse_args():
@@ -205,6 +205,23 @@ class ClockSampler:
         return out
 
 
+# ------------------------------------------------------------------------------------- ranks
+def max_over_ranks(ms, device, world):
+    """Slowest rank's time: the job is as fast as its slowest replica."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_throughput(units_per_rank, world, ms_per_step):
+    """Every rank processes its own batch of the same size (weak scaling): units of all ranks per second."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
 # ------------------------------------------------------------------------------------- GPU arm
 def run_sharpv(args):
     import torch
@@ -369,12 +386,9 @@ def run_sharpv(args):
     stage_ms = {name: timed_launches(fn, stage_n) for name, fn in stages}
     clocks = sampler.stop() if sampler else None
 
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dev, world)
     ms_per_step = total_ms / args.steps
-    value = world * NV / (ms_per_step * 1e-3)
+    value = whole_job_throughput(NV, world, ms_per_step)
 
     # ---- end to end: inputs start in pinned host memory, results are read back every step
     h_tokens, h_hidden = pinned(wl.tokens), pinned(wl.hidden)
@@ -404,10 +418,7 @@ def run_sharpv(args):
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, dev, world)
     h2d = h_tokens.numel() * h_tokens.element_size() + h_hidden.numel() * h_hidden.element_size()
     d2h = (h_idx.numel() + h_pos.numel() + h_cnt.numel() + h_kso.numel()) * 4
 
@@ -460,7 +471,7 @@ def run_sharpv(args):
         "kv_compaction_GBps": kernels["compact"]["GBps"],
         "roofline": roofline, "kernels": kernels,
         "cpu_baseline": cpu,
-        "e2e": {"value": world * NV / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+        "e2e": {"value": whole_job_throughput(NV, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "note": "tokens and hidden state copied from pinned host memory every step, kept-index lists "
                         "read back; the K/V cache is device-resident model state"},

@@ -104,14 +104,14 @@ __device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
     return d;
 }
 // one 32-bit word of two bf16 -> the two exact fp32 values (a bf16 is the upper half of an fp32):
-// two byte permutes written straight into the halves of the 64-bit result
+// one multiply and one mask, on different pipes, written straight into the halves of the result
 __device__ __forceinline__ f32x2 widen_bf16x2(uint32_t w) {
     f32x2 r;
     asm("{\n\t.reg .b32 lo, hi;\n\t"
-        "prmt.b32 lo, %1, %2, 0x1044;\n\t"
-        "prmt.b32 hi, %1, %2, 0x3244;\n\t"
+        "mul.lo.u32 lo, %1, 65536;\n\t"          // low element: shift up (multiply pipe)
+        "and.b32 hi, %1, 0xffff0000;\n\t"        // high element: mask (logic pipe)
         "mov.b64 %0, {lo, hi};\n\t}"
-        : "=l"(r) : "r"(w), "r"(0u));
+        : "=l"(r) : "r"(w));
     return r;
 }
 __device__ __forceinline__ f32x2 pair_f32(uint32_t lo, uint32_t hi) {
@@ -338,6 +338,7 @@ struct Pass {
         if (*abort_flag) return false;
         if (tid == 0 && q + pp.nbuf < Q) issue_load(q + pp.nbuf);
         // column sums over the 64 row groups: fixed order, two levels
+#pragma unroll
         for (int e = tid; e < 4 * SE; e += kThreads) {
             const int col = e % SE, quarter = e / SE;
             float sum = 0.f;

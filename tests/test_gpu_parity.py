@@ -359,3 +359,79 @@ def test_strided_token_rows():
     torch.cuda.synchronize()
     n = int(sa["num_kept"].item())
     assert torch.equal(sa["tokens"][:n], sb["tokens"][:n])
+
+
+# ------------------------------------------------------------------------------------------------
+# full-size workloads in the launch configuration the benchmark times
+# ------------------------------------------------------------------------------------------------
+def _device_kv(wl, seed):
+    """N(0,1) K/V drawn on the device with torch's generator (values never influence a decision)."""
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+    dt = torch.float32 if wl.dtype == W.F32 else torch.bfloat16
+    kv = torch.empty(wl.kv_shape(), dtype=dt, device="cuda")
+    for l in range(wl.num_layers):
+        kv[l] = torch.randn(wl.kv_shape()[1:], dtype=torch.float32, device="cuda", generator=gen).to(dt)
+    return kv
+
+
+@pytest.mark.parametrize("name", ["ragged_batch", "long_video"])
+def test_full_size_workloads(name):
+    """The 16-video ragged batch (424 frames) and the 256-frame video at their full sizes: scores,
+    budgets and kept sets element by element against the oracle; compacted K/V (4.8 GB / 2.9 GB) on
+    sampled planes and rows plus properties that hold for every plane."""
+    wl = W.PRESETS[name]()
+    W.fill_tokens(wl)
+    W.fill_hidden(wl)
+    dw = DeviceWorkload(wl)
+    F, f, T, M = wl.total_frames, wl.f, wl.total_seq_tokens, 0.788
+    o = orc.score_frames(wl.tokens, wl.video_frame_offsets, f, nthreads=NT)
+    g = sv.sharpv_score_frames(dw.tokens, dw.video_frame_offsets, F, f, want_spatial=True, want_temporal=True)
+    torch.cuda.synchronize()
+    for key in ("spatial", "temporal", "importance", "ratio"):
+        e = rel_err(to_host(g[key]), o[key])
+        assert e <= TIGHT_TOL, f"{key}: rel err {e}"
+    k_gpu = to_host(g["k"])
+    assert len(check_budgets(k_gpu, o, f)) <= max(1, F // 50)
+    sel = sv.sharpv_select_tokens(g["importance"], g["k"], F, f, tokens=dw.tokens)
+    torch.cuda.synchronize()
+    n = int(sel["num_kept"].item())
+    assert n == int(k_gpu.sum())
+    idx = to_host(sel["kept_index"])[:n]
+    exempt = check_kept_sets(idx, to_host(sel["kept_offsets"]), o["importance"], k_gpu, f, orc.select_tokens)
+    assert exempt <= max(2, n // 1000)
+    rows = np.random.default_rng(80).choice(n, size=min(n, 512), replace=False)
+    got = sel["tokens"][torch.from_numpy(rows).cuda()]
+    np.testing.assert_array_equal(to_host(got), wl.tokens[idx[rows]])
+
+    oc = orc.kv_calibrate_prune(wl.hidden, wl.tokens, wl.seq_offsets, wl.vis_begin, wl.vis_count, wl.vis_offsets,
+                                M, nthreads=NT)
+    gc = sv.sharpv_kv_calibrate_prune(dw.hidden, dw.tokens, dw.seq_offsets, dw.vis_begin, dw.vis_count,
+                                      dw.vis_offsets, T, M=M)
+    torch.cuda.synchronize()
+    assert rel_err(to_host(gc["cos"])[:wl.n_visual], oc["cos"]) <= TIGHT_TOL
+    kso = to_host(gc["kept_seq_offsets"])
+    nk = int(kso[-1])
+    kept = to_host(gc["kept_pos"])[:nk]
+    sym = np.setxor1d(kept, oc["kept_pos"])
+    assert sym.size <= max(2, wl.n_visual // 1000)
+    if sym.size == 0:
+        np.testing.assert_array_equal(kso, oc["kept_seq_offsets"])
+
+    kv = _device_kv(wl, 81)
+    dst = torch.zeros_like(kv)
+    sv.sharpv_kv_compact(kv, dst, gc["kept_pos"], gc["kept_seq_offsets"], capacity=T)
+    torch.cuda.synchronize()
+    L, _, H, _, Dh = wl.kv_shape()
+    rng = np.random.default_rng(82)
+    planes = {(0, 0, 0), (L - 1, 1, H - 1)} | {(int(rng.integers(L)), int(rng.integers(2)), int(rng.integers(H)))
+                                               for _ in range(6)}
+    for (l, kvi, h) in planes:                       # sampled planes against the oracle, whole plane
+        src_plane = to_host(kv[l, kvi, h])[None, None, None]          # [1, 1, 1, T, Dh] ... one-plane cache
+        src5 = np.ascontiguousarray(np.broadcast_to(src_plane, (1, 2, 1, T, Dh)))
+        expect = orc.kv_compact(src5, kept)[0, 0, 0]
+        np.testing.assert_array_equal(to_host(dst[l, kvi, h]), expect)
+    # every plane: the kept prefix equals the gathered source rows, the rest is untouched
+    kept_d = gc["kept_pos"][:nk].long()
+    assert torch.equal(dst[:, :, :, :nk].view(torch.int16), kv[:, :, :, kept_d].view(torch.int16))
+    assert int(dst[:, :, :, nk:].view(torch.int16).abs().max().item()) == 0
