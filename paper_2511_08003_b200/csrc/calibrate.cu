@@ -34,6 +34,7 @@ calibrate_cos_kernel(const char* __restrict__ hidden, int64_t hidden_row_bytes,
     constexpr int P = E::kPerVec;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t p = (int64_t)blockIdx.x * kRowsPerCta + warp;
+    cudaGridDependencySynchronize();        // hidden states and counters come from earlier work on the stream
     if (p >= T) return;
     const int b = upper_segment(seq_offsets, num_seqs, (int)p);
     const int64_t local = p - __ldg(seq_offsets + b) - __ldg(vis_begin + b);
@@ -200,15 +201,16 @@ static sharpv_status calibrate_impl(
     // the per-chunk counts are accumulated with atomics and must start at zero
     if (cudaMemsetAsync(chunk_counts, 0, sizeof(int32_t) * (size_t)chunks, stream) != cudaSuccess)
         return SHARPV_ERR_CUDA;
-    if (dtype == SHARPV_F32)
-        calibrate_cos_kernel<SHARPV_F32><<<ctas, 256, 0, stream>>>(
-            (const char*)hidden, ld_hidden * eb, (const char*)visual, ld_visual * eb, nvec, num_seqs, seq_offsets,
-            vis_begin, vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, flags, chunk_counts);
-    else
-        calibrate_cos_kernel<SHARPV_BF16><<<ctas, 256, 0, stream>>>(
-            (const char*)hidden, ld_hidden * eb, (const char*)visual, ld_visual * eb, nvec, num_seqs, seq_offsets,
-            vis_begin, vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, flags, chunk_counts);
-    if (cudaGetLastError() != cudaSuccess) return SHARPV_ERR_CUDA;
+    {
+        auto kern = dtype == SHARPV_F32 ? calibrate_cos_kernel<SHARPV_F32> : calibrate_cos_kernel<SHARPV_BF16>;
+        if (launch_dependent(kern, dim3(ctas), dim3(256), 0, stream, (const char*)hidden, ld_hidden * eb,
+                             (const char*)visual, ld_visual * eb, nvec, (int)num_seqs, seq_offsets, vis_begin,
+                             vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, flags,
+                             chunk_counts) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return SHARPV_ERR_CUDA;
+        }
+    }
     if (launch_dependent(write_kept_kernel, dim3(chunks), dim3(kChunk), 0, stream, (const uint8_t*)flags,
                          (const int32_t*)chunk_counts, total_seq_tokens, num_seqs, seq_offsets, capacity,
                          out_kept_pos, out_kept_seq_offsets, status_word) != cudaSuccess) {

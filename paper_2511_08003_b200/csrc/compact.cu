@@ -28,6 +28,7 @@ __global__ void __launch_bounds__(kCompactThreads)
 kv_compact_kernel(const char* __restrict__ src, char* __restrict__ dst, PlaneGeom g, int planes,
                   const int32_t* __restrict__ kept_pos, const int32_t* __restrict__ n_kept_ptr,
                   int64_t capacity, int32_t* status_word) {
+    cudaGridDependencySynchronize();        // the index list and the cache come from earlier work on the stream
     const int64_t n_all = __ldg(n_kept_ptr);
     if (blockIdx.x == 0 && threadIdx.x == 0 && n_all > capacity) report(status_word, SHARPV_ERR_CAPACITY);
     const int64_t n = min(n_all, capacity);
@@ -123,7 +124,11 @@ extern "C" sharpv_status sharpv_kv_compact(
     const int64_t max_tiles = (capacity + tile_rows - 1) / tile_rows * planes;
     const int64_t want = (int64_t)sms * kCompactCtasPerSm;
     const unsigned grid = (unsigned)(max_tiles < want ? max_tiles : want);
-    kv_compact_kernel<kCompactUnroll><<<grid, kCompactThreads, 0, (cudaStream_t)cuda_stream>>>(
-        (const char*)kv_src, (char*)kv_dst, g, planes, kept_pos, kept_seq_offsets + num_seqs, capacity, status_word);
+    if (launch_dependent(kv_compact_kernel<kCompactUnroll>, dim3(grid), dim3(kCompactThreads), 0,
+                         (cudaStream_t)cuda_stream, (const char*)kv_src, (char*)kv_dst, g, planes, kept_pos,
+                         kept_seq_offsets + num_seqs, capacity, status_word) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SHARPV_ERR_CUDA;
+    }
     return launch_status();
 }

@@ -404,6 +404,7 @@ score_pass_kernel(const __grid_constant__ CUtensorMap tmap, const FusedParams p,
 
     // let the finaliser's CTAs be scheduled as soon as SMs free up; they wait for this whole grid
     cudaTriggerProgrammaticLaunchCompletion();
+    cudaGridDependencySynchronize();        // the tokens come from earlier work on the stream
     const int64_t U = (int64_t)p.nsl * p.F;
     const int64_t u0 = U * blockIdx.x / gridDim.x;
     const int64_t u1 = U * (blockIdx.x + 1) / gridDim.x;
@@ -641,8 +642,11 @@ sharpv_status launch(const FusedScoreArgs& a, const CUtensorMap& tmap, FusedPara
     }
     const int64_t units = (int64_t)p.nsl * a.F;
     const unsigned grid = (unsigned)(units < sms ? units : sms);
-    score_pass_kernel<DT><<<grid, kThreads, smem, a.stream>>>(tmap, p, a.status_word);
-    if (cudaGetLastError() != cudaSuccess) return SHARPV_ERR_CUDA;
+    if (launch_dependent(score_pass_kernel<DT>, dim3(grid), dim3(kThreads), smem, a.stream, tmap, p,
+                         a.status_word) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SHARPV_ERR_CUDA;
+    }
 
     // the finaliser starts while the pass drains and waits for it with cudaGridDependencySynchronize
     if (launch_dependent(score_finalize_kernel<DT>, dim3((unsigned)a.F), dim3(kFinThreads), 0, a.stream, p) !=

@@ -52,6 +52,7 @@ select_frame_kernel(const float* __restrict__ importance, const int32_t* __restr
     const int t = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float* imp = importance + (int64_t)t * f;
+    cudaGridDependencySynchronize();        // scores and budgets come from earlier work on the stream
 
     // exclusive scan of the (clamped) budgets: every CTA adds up the frames in front of it
     int part = 0;
@@ -217,9 +218,12 @@ sharpv_status select_impl(int mode, const float* importance, const int32_t* k, f
             return SHARPV_ERR_CUDA;
         return SHARPV_OK;
     }
-    select_frame_kernel<<<F, kSelectThreads, (size_t)f * 4, stream>>>(
-        importance, budgets, F, f, capacity, mode, K, out_kept_offsets, out_num_kept, out_kept_index, status_word);
-    if (cudaGetLastError() != cudaSuccess) return SHARPV_ERR_CUDA;
+    if (launch_dependent(select_frame_kernel, dim3((unsigned)F), dim3(kSelectThreads), (size_t)f * 4, stream,
+                         importance, budgets, (int)F, (int)f, capacity, mode, K, out_kept_offsets, out_num_kept,
+                         out_kept_index, status_word) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SHARPV_ERR_CUDA;
+    }
     if (out_tokens && capacity > 0) {
         const int64_t rows = capacity < (int64_t)F * f ? capacity : (int64_t)F * f;
         const int nvec = d * eb / 16;
