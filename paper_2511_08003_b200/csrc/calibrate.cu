@@ -19,10 +19,10 @@ constexpr int kChunk = 256;             // packed positions per chunk of the fla
 __host__ __device__ inline size_t ws_flags_bytes(int64_t T) { return ((size_t)T + 255) / 256 * 256; }
 __host__ __device__ inline int64_t num_chunks(int64_t T) { return (T + kChunk - 1) / kChunk; }
 
-constexpr int kRowsPerCta = 8;          // one packed position per warp
+constexpr int kRowsPerCta = 4;          // one packed position per warp; small CTAs balance the SMs
 
 template <int DT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kRowsPerCta * 32)
 calibrate_cos_kernel(const char* __restrict__ hidden, int64_t hidden_row_bytes,
                      const char* __restrict__ visual, int64_t visual_row_bytes, int nvec,
                      int num_seqs, const int32_t* __restrict__ seq_offsets,
@@ -99,30 +99,33 @@ write_kept_kernel(const uint8_t* __restrict__ flags, const int32_t* __restrict__
     __shared__ int s_base;
     const int c = blockIdx.x;
     cudaGridDependencySynchronize();        // flags and chunk counts come from the kernel in front
-    // kept positions before this chunk: fixed-order sum of the earlier chunk counts
+    // all global loads of this thread are issued up front: one memory round trip, not three
+    const int64_t p = (int64_t)c * kChunk + threadIdx.x;
+    const int keep = p < T ? flags[p] : 0;
     int part = 0;
     for (int i = threadIdx.x; i < c; i += kChunk) part += chunk_counts[i];
+    int seq_first = -1, seq_last = -1;      // sequences that start at p: [seq_first, seq_last]
+    if (p < T) {
+        int b = upper_segment(seq_offsets, num_seqs, (int)p);
+        if (__ldg(seq_offsets + b) == (int)p) {
+            seq_last = b;
+            while (b > 0 && __ldg(seq_offsets + b - 1) == (int)p) --b;
+            seq_first = b;
+        }
+    }
+    // kept positions before this chunk: fixed-order sum of the earlier chunk counts
     int total_before;
     block_exclusive_scan<kChunk>(part, sm, total_before);
     if (threadIdx.x == 0) s_base = total_before;
     __syncthreads();
     const int base = s_base;
 
-    const int64_t p = (int64_t)c * kChunk + threadIdx.x;
-    const int keep = p < T ? flags[p] : 0;
     int chunk_total;
     const int rank = block_exclusive_scan<kChunk>(keep, sm, chunk_total);
     const int64_t j = (int64_t)base + rank;
     if (keep && j < capacity) out_kept_pos[j] = (int32_t)p;
+    for (int b = seq_first; b >= 0 && b <= seq_last; ++b) out_kept_seq_offsets[b] = (int32_t)j;
 
-    // sequences that start at this position (several when some are empty)
-    if (p < T) {
-        int b = upper_segment(seq_offsets, num_seqs, (int)p);
-        while (b >= 0 && __ldg(seq_offsets + b) == (int)p) {
-            out_kept_seq_offsets[b] = (int32_t)j;
-            --b;
-        }
-    }
     if (c == gridDim.x - 1 && threadIdx.x == 0) {
         const int64_t total = (int64_t)base + chunk_total;
         // trailing empty sequences and the end marker
@@ -203,7 +206,7 @@ static sharpv_status calibrate_impl(
         return SHARPV_ERR_CUDA;
     {
         auto kern = dtype == SHARPV_F32 ? calibrate_cos_kernel<SHARPV_F32> : calibrate_cos_kernel<SHARPV_BF16>;
-        if (launch_dependent(kern, dim3(ctas), dim3(256), 0, stream, (const char*)hidden, ld_hidden * eb,
+        if (launch_dependent(kern, dim3(ctas), dim3(kRowsPerCta * 32), 0, stream, (const char*)hidden, ld_hidden * eb,
                              (const char*)visual, ld_visual * eb, nvec, (int)num_seqs, seq_offsets, vis_begin,
                              vis_count, vis_offsets, total_seq_tokens, total_visual, M, out_cos, flags,
                              chunk_counts) != cudaSuccess) {

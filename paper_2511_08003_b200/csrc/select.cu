@@ -45,8 +45,9 @@ select_frame_kernel(const float* __restrict__ importance, const int32_t* __restr
                     int64_t capacity, int mode, float K, int32_t* __restrict__ kept_offsets,
                     int32_t* __restrict__ num_kept, int32_t* __restrict__ out_kept_index, int32_t* status_word) {
     extern __shared__ uint32_t keys[];                 // [f]
-    __shared__ int hist[256];
+    __shared__ int hist[4][256];                       // one histogram per byte pass, cleared once
     __shared__ int scan_sm[kSelectThreads / 32 + 1];
+    __shared__ int off_sm[kSelectThreads / 32];
     __shared__ int s_digit, s_remaining;
 
     const int t = blockIdx.x;
@@ -54,16 +55,23 @@ select_frame_kernel(const float* __restrict__ importance, const int32_t* __restr
     const float* imp = importance + (int64_t)t * f;
     cudaGridDependencySynchronize();        // scores and budgets come from earlier work on the stream
 
-    // exclusive scan of the (clamped) budgets: every CTA adds up the frames in front of it
+    // this frame's offset: the (clamped) budgets of the frames in front of it, added in a fixed order
     int part = 0;
     for (int i = tid; i < t; i += kSelectThreads) part += min(max(k[i], 0), f);
-    int before;
-    block_exclusive_scan<kSelectThreads>(part, scan_sm, before);
+    const int kt_raw = k[t];
+    for (int i = tid; i < f; i += kSelectThreads) keys[i] = mode == 0 ? order_key(imp[i]) : (imp[i] > K ? 1u : 0u);
+    for (int i = tid; i < 4 * 256; i += kSelectThreads) (&hist[0][0])[i] = 0;
+    part = warp_sum_int(part);
+    if (lane == 0) off_sm[warp] = part;
+    __syncthreads();
+    int before = 0;
+#pragma unroll
+    for (int i = 0; i < kSelectThreads / 32; ++i) before += off_sm[i];
     const int64_t out_base = before;
     if (tid == 0) {
         kept_offsets[t] = before;
         if (t == F - 1) {
-            const int total = before + min(max(k[t], 0), f);
+            const int total = before + min(max(kt_raw, 0), f);
             kept_offsets[F] = total;
             if (num_kept) *num_kept = total;
             if ((int64_t)total > capacity) report(status_word, SHARPV_ERR_CAPACITY);
@@ -74,29 +82,26 @@ select_frame_kernel(const float* __restrict__ importance, const int32_t* __restr
     int remaining = 0;
     bool keep_all = false;
     if (mode == 0) {
-        const int kt = min(max(k[t], 0), f);
+        const int kt = min(max(kt_raw, 0), f);
         if (kt == 0) return;
         keep_all = kt == f;
-        for (int i = tid; i < f; i += kSelectThreads) keys[i] = order_key(imp[i]);
-        __syncthreads();
         if (!keep_all) {
             // radix select, most significant byte first: after the four passes `prefix` is the
             // k-th largest key and `remaining` says how many keys equal to it are still owed
             uint32_t prefix = 0, mask = 0;
             remaining = kt;
-            for (int shift = 24; shift >= 0; shift -= 8) {
-                for (int i = tid; i < 256; i += kSelectThreads) hist[i] = 0;
-                __syncthreads();
+            int pass = 0;
+            for (int shift = 24; shift >= 0; shift -= 8, ++pass) {
                 for (int i = tid; i < f; i += kSelectThreads) {
                     const uint32_t key = keys[i];
-                    if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+                    if ((key & mask) == prefix) atomicAdd(&hist[pass][(key >> shift) & 255u], 1);
                 }
                 __syncthreads();
                 if (warp == 0) {
                     const int top = 255 - lane * 8;    // lane 0 owns the 8 largest digits
                     int c[8], sum = 0;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) { c[j] = hist[top - j]; sum += c[j]; }
+                    for (int j = 0; j < 8; ++j) { c[j] = hist[pass][top - j]; sum += c[j]; }
                     int inc = sum;
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) {
@@ -122,65 +127,53 @@ select_frame_kernel(const float* __restrict__ importance, const int32_t* __restr
             }
             kth = prefix;
         }
-    } else {
-        // threshold variant: key 1 for kept, 0 otherwise; "greater than 0" keeps them
-        for (int i = tid; i < f; i += kSelectThreads) keys[i] = imp[i] > K ? 1u : 0u;
-        __syncthreads();
-        kth = 0;
-        remaining = 0;
     }
+    // threshold variant: keys are 1 (kept) or 0, kth = 0, remaining = 0: "greater than 0" keeps them
 
-    // index-ordered pass: keys above the k-th are kept; among keys equal to it the first
-    // `remaining` in index order are kept
-    int carry_eq = 0, carry_keep = 0;
+    // index-ordered pass: keys above the k-th are kept; among keys equal to it the first `remaining`
+    // in index order are kept.  One scan carries both counts (low half: greater, high half: equal).
+    int carry = 0;
     for (int base = 0; base < f; base += kSelectThreads) {
         const int i = base + tid;
         const bool valid = i < f;
         const uint32_t key = valid ? keys[i] : 0u;
-        bool keep;
-        if (keep_all) {
-            keep = valid;
-        } else {
-            const bool gt = valid && key > kth;
-            const int eq = (valid && key == kth && remaining > 0) ? 1 : 0;
-            int tot_eq;
-            const int eq_rank = carry_eq + block_exclusive_scan<kSelectThreads>(eq, scan_sm, tot_eq);
-            carry_eq += tot_eq;
-            keep = gt || (eq && eq_rank < remaining);
-        }
-        int tot_keep;
-        const int pos = carry_keep + block_exclusive_scan<kSelectThreads>(keep ? 1 : 0, scan_sm, tot_keep);
-        carry_keep += tot_keep;
-        if (keep) {
-            const int64_t j = out_base + pos;
+        const bool gt = valid && (keep_all || key > kth);
+        const bool eq = valid && !keep_all && key == kth && remaining > 0;
+        int total;
+        const int pre = carry + block_exclusive_scan<kSelectThreads>((gt ? 1 : 0) | (eq ? 1 << 16 : 0), scan_sm, total);
+        carry += total;
+        const int gt_before = pre & 0xffff, eq_before = pre >> 16;
+        if (gt || (eq && eq_before < remaining)) {
+            const int64_t j = out_base + gt_before + min(eq_before, remaining);
             if (j < capacity) out_kept_index[j] = t * f + i;
         }
     }
 }
 
+// one warp per half row, up to eight 128-bit loads in flight per lane
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const char* __restrict__ src, int64_t src_row_bytes, int nvec,
                    const int32_t* __restrict__ index, const int32_t* __restrict__ count_ptr,
                    int64_t capacity, char* __restrict__ dst, int64_t dst_row_bytes) {
     cudaGridDependencySynchronize();        // the index list comes from the kernel in front
     const int lane = threadIdx.x & 31;
-    const int64_t j = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int64_t w = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int64_t j = w >> 1;
     const int64_t n = min((int64_t)__ldg(count_ptr), capacity);
     if (j >= n) return;
+    const int half = (nvec + 1) >> 1;
+    const int v0 = (int)(w & 1) * half, v1 = min(nvec, v0 + half);
     const char* s = src + (int64_t)__ldg(index + j) * src_row_bytes;
     char* o = dst + j * dst_row_bytes;
-    int v = lane;
-    for (; v + 96 < nvec; v += 128) {
-        uint4 r0 = ld_stream(s + (int64_t)v * 16);
-        uint4 r1 = ld_stream(s + (int64_t)(v + 32) * 16);
-        uint4 r2 = ld_stream(s + (int64_t)(v + 64) * 16);
-        uint4 r3 = ld_stream(s + (int64_t)(v + 96) * 16);
-        st_stream(o + (int64_t)v * 16, r0);
-        st_stream(o + (int64_t)(v + 32) * 16, r1);
-        st_stream(o + (int64_t)(v + 64) * 16, r2);
-        st_stream(o + (int64_t)(v + 96) * 16, r3);
+    for (int v = v0 + lane; v < v1; v += 256) {
+        uint4 r[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (v + 32 * u < v1) r[u] = ld_stream(s + (int64_t)(v + 32 * u) * 16);
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (v + 32 * u < v1) st_stream(o + (int64_t)(v + 32 * u) * 16, r[u]);
     }
-    for (; v < nvec; v += 32) st_stream(o + (int64_t)v * 16, ld_stream(s + (int64_t)v * 16));
 }
 
 sharpv_status select_impl(int mode, const float* importance, const int32_t* k, float K, int32_t F, int32_t f,
@@ -227,7 +220,7 @@ sharpv_status select_impl(int mode, const float* importance, const int32_t* k, f
     if (out_tokens && capacity > 0) {
         const int64_t rows = capacity < (int64_t)F * f ? capacity : (int64_t)F * f;
         const int nvec = d * eb / 16;
-        if (launch_dependent(gather_rows_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, stream,
+        if (launch_dependent(gather_rows_kernel, dim3((unsigned)((2 * rows + 7) / 8)), dim3(256), 0, stream,
                              (const char*)tokens, ld_tokens * eb, nvec, (const int32_t*)out_kept_index,
                              (const int32_t*)(out_kept_offsets + F), capacity, (char*)out_tokens,
                              (int64_t)d * eb) != cudaSuccess) {
