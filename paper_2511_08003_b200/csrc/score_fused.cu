@@ -4,16 +4,17 @@
 // the f x 256-byte tile of frame t.  Persistent CTAs (one per SM) each take a contiguous range of
 // units in (slice-major, frame-minor) order, so a CTA walks consecutive frames of one slice.
 //
-//   score_pass_kernel      TMA brings the next tiles into a ring of shared-memory buffers.  Each
-//       thread keeps its part of the previous frame's tile in registers (4 rows x two 16-byte
-//       vectors) and visits the new tile once: column sums (they give this slice of the frame
-//       mean, the whole frame column being inside the tile), ||a||^2, ||a-b||^2 against the
-//       previous frame, and <b, mean(b)> for the previous frame, whose mean is known by now.
-//       The new rows then replace the old ones in the same registers.  Per-row partial sums of
-//       the slice go to a small workspace.  The only wait is on the CTA's own TMA loads and it
-//       is bounded.
-//   score_finalize_kernel  one CTA per frame, launched with programmatic dependent launch so that
-//       its start-up overlaps the tail of the pass: adds the slices in a fixed order and writes
+//   score_pass_kernel      640 threads in two roles that only meet through mbarriers:
+//       column warps (4)   issue the TMA loads that fill a ring of tile buffers, add up the columns
+//                          of each tile (the whole frame column is inside the tile, so this is the
+//                          slice of the frame mean) and publish the mean one tile ahead of the rows;
+//       row warps (16)     keep their part of the previous frame's tile in registers (4 rows x two
+//                          16-byte vectors per thread), visit each new tile once for ||a||^2,
+//                          ||a - mean||^2 and ||a - b||^2 with packed fp32 FMAs, overwrite the old
+//                          rows in place and write one record of partial sums per row and slice.
+//       Every wait is on the CTA's own barriers and is bounded.
+//   score_finalize_kernel  one CTA per frame, launched as a programmatic dependent so that its
+//       start-up overlaps the tail of the pass: adds the slices in a fixed order and writes
 //       S, T, I, the ratio and the budget of the frame.
 #include <cuda.h>
 
@@ -24,18 +25,24 @@ namespace sharpv {
 namespace {
 
 constexpr int kSliceBytes = 256;
-constexpr int kThreads = 512;           // 16 warps; a warp = 4 row groups x 8 lanes (two vectors per lane)
-constexpr int kRowGroups = kThreads / 8;
-constexpr int kRows = 4;                // row slots per thread: frames of up to 256 tokens
+constexpr int kRowWarps = 16;           // a row warp = 4 row groups x 8 lanes (two vectors per lane)
+constexpr int kColWarps = 4;            // 128 threads = 16 vector columns x 8 row groups
+constexpr int kRowThreads = kRowWarps * 32;
+constexpr int kColThreads = kColWarps * 32;
+constexpr int kThreads = kRowThreads + kColThreads;
+constexpr int kColGroups = kColThreads / 16;
+constexpr int kRows = 4;                // row slots per row-warp thread: frames of up to 256 tokens
 constexpr int kMaxTokensFused = 256;
+constexpr int kNBuf = 3;                // tile buffers in the ring
 constexpr int kSmemBudget = 227 * 1024;
-constexpr uint32_t kSpinLimit = 1u << 22;      // polls of one mbarrier before a wait gives up
+constexpr uint32_t kSpinLimit = 1u << 24;      // polls of one mbarrier before a wait gives up
+constexpr long long kSpinClocks = 2000000000ll; // ... or about one second of SM clock
 constexpr int kFinThreads = 1024;
 
 struct FusedParams {
     const char* tokens;
     int64_t row_bytes_ld;
-    int F, f, d, nsl, nvec, nbuf;
+    int F, f, d, nsl, nvec;
     int num_videos;
     const int32_t* video_frame_offsets;
     float w;
@@ -43,7 +50,7 @@ struct FusedParams {
     float *out_I, *out_S, *out_T, *out_ratio;
     int32_t* out_k;
     float* mean;            // [F, d]
-    float4* part;           // [F, nsl, f]: (||a||^2, ||a-b||^2, ||b||^2, <a, mean>) of the slice
+    float4* part;           // [F, nsl, f]: (||a||^2, ||a-m||^2, ||a-b||^2, ||b||^2) of the slice
     uint32_t tile_bytes, tile_stride;
 };
 
@@ -51,6 +58,9 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
@@ -64,10 +74,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// bounded wait: false when the limit ran out
+// bounded wait: false when the limit ran out (a poll count and, every 256 polls, about a second of
+// SM clock, whichever comes first)
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t i = 1; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 0 && clock64() - t0 > kSpinClocks) return false;
+    }
     return false;
 }
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -154,66 +169,202 @@ __device__ __forceinline__ bool frame_is_first(const int32_t* vfo, int num_video
     return __ldg(vfo + b) == t;
 }
 
+// Shared-memory layout of one CTA.
 template <int DT>
-struct Pass {
-    using E = Elem<DT>;
-    static constexpr int P = E::kPerVec;                    // elements per 16-byte vector
-    static constexpr int H = P / 2;                         // packed pairs per vector
-    static constexpr int SE = kSliceBytes / E::kBytes;      // elements per slice row
-
-    const CUtensorMap* tmap;
-    const FusedParams* p;
-    unsigned char* tiles;
-    float* cs;              // [kRowGroups][SE] column sums of each row group
-    float* cs2;             // [4][SE]
-    float* mean_s;          // [SE]
-    uint64_t* bars;         // [nbuf]
+struct Smem {
+    static constexpr int SE = kSliceBytes / Elem<DT>::kBytes;       // elements per slice row
+    unsigned char* tiles;       // [kNBuf][tile_stride]
+    float* cs;                  // [kColGroups][SE] column sums of each row group of the column warps
+    float* mean_s;              // [2][SE] frame-mean slice of the tiles, alternating
+    uint64_t* full;             // [kNBuf] tile landed (TMA)
+    uint64_t* empty;            // [kNBuf] tile released by all 20 warps
+    uint64_t* mean_full;        // [2] mean published by the column warps
+    uint64_t* mean_empty;       // [2] mean read by all 16 row warps
     volatile int* abort_flag;
-    int Q, halo;
-    int load_s, load_t;     // (slice, frame) of the next tile to request (thread 0 only)
 
-    // per-thread state carried from frame to frame
-    uint4 prev[kRows][2];   // previous frame's rows of this thread (two vectors each)
-    f32x2 mprev[2][H];      // previous frame's mean over this thread's columns
-    float bb[kRows];        // this thread's share of ||previous row||^2
-
-    int tid, warp, g, j, rgid;
-
-    // requests tile q; tiles are requested in unit order, so (load_s, load_t) just advances
-    __device__ __forceinline__ void issue_load(int q) {
-        const FusedParams& pp = *p;
-        const int slot = q % pp.nbuf;
-        uint64_t* bar = bars + slot;
-        mbar_expect_tx(bar, pp.tile_bytes);
-        tma_load_2d(tiles + (size_t)slot * pp.tile_stride, tmap, load_s * kSliceBytes, load_t * pp.f, bar);
-        if (++load_t == pp.F) { load_t = 0; ++load_s; }
+    __device__ __forceinline__ Smem(unsigned char* base, uint32_t tile_stride) {
+        tiles = base;
+        cs = reinterpret_cast<float*>(base + (size_t)kNBuf * tile_stride);
+        mean_s = cs + kColGroups * SE;
+        full = reinterpret_cast<uint64_t*>(mean_s + 2 * SE);
+        empty = full + kNBuf;
+        mean_full = empty + kNBuf;
+        mean_empty = mean_full + 2;
+        abort_flag = reinterpret_cast<volatile int*>(mean_empty + 2);
     }
+    static size_t fixed_bytes() { return (size_t)(kColGroups * SE + 2 * SE) * 4 + (2 * kNBuf + 4) * 8 + 16; }
+};
 
-    __device__ __forceinline__ const unsigned char* wait_tile(int slot, uint32_t phase) const {
-        if (!mbar_wait(bars + slot, phase)) *abort_flag = 1;
-        return tiles + (size_t)slot * p->tile_stride;
+// where a CTA stands in its range of units
+struct Walk {
+    int s, t;           // slice and frame of the current unit
+    int vid, next_start;
+    bool is_first;      // frame t opens a video
+
+    __device__ __forceinline__ void start(const FusedParams& p, int64_t u0) {
+        s = (int)(u0 / p.F);
+        t = (int)(u0 % p.F);
+        vid = upper_segment(p.video_frame_offsets, p.num_videos, t);
+        is_first = __ldg(p.video_frame_offsets + vid) == t;
+        next_start = __ldg(p.video_frame_offsets + vid + 1);
     }
+    // advances to the next unit; returns true when it starts a new slice
+    __device__ __forceinline__ bool step(const FusedParams& p) {
+        if (++t == p.F) {
+            t = 0;
+            ++s;
+            vid = upper_segment(p.video_frame_offsets, p.num_videos, 0);
+            next_start = __ldg(p.video_frame_offsets + vid + 1);
+            is_first = true;
+            return true;
+        }
+        is_first = false;
+        while (t >= next_start && vid + 1 < p.num_videos) {         // skips videos without frames
+            ++vid;
+            is_first = true;
+            next_start = __ldg(p.video_frame_offsets + vid + 1);
+        }
+        return false;
+    }
+};
 
-    __device__ __forceinline__ static void to_pairs(const uint4& v, f32x2 (&o)[H]) {
-        if (DT == SHARPV_BF16) {
-            o[0] = widen_bf16x2(v.x); o[1] = widen_bf16x2(v.y);
-            o[H - 2] = widen_bf16x2(v.z); o[H - 1] = widen_bf16x2(v.w);
+template <int DT>
+__device__ __forceinline__ void widen_pairs(const uint4& v, f32x2 (&o)[Elem<DT>::kPerVec / 2]) {
+    constexpr int H = Elem<DT>::kPerVec / 2;
+    if (DT == SHARPV_BF16) {
+        o[0] = widen_bf16x2(v.x); o[1] = widen_bf16x2(v.y);
+        o[H - 2] = widen_bf16x2(v.z); o[H - 1] = widen_bf16x2(v.w);
+    } else {
+        o[0] = pair_f32(v.x, v.y); o[H - 1] = pair_f32(v.z, v.w);
+    }
+}
+
+// barrier 1 over the column warps with an OR of `flag`: every thread gets the same answer
+__device__ __forceinline__ bool column_any(bool flag) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, 1, %2, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out) : "r"((uint32_t)flag), "n"(kColThreads) : "memory");
+    return out != 0;
+}
+
+// ---------------------------------------------------------------------------------------
+// column warps: TMA producer, column sums, frame mean
+// ---------------------------------------------------------------------------------------
+template <int DT>
+__device__ __forceinline__ void column_role(const CUtensorMap* tmap, const FusedParams& p, Smem<DT>& sm, int64_t u0,
+                                            int n_units, int halo, int ctid) {
+    using E = Elem<DT>;
+    constexpr int P = E::kPerVec, H = P / 2, SE = Smem<DT>::SE;
+    const int Q = n_units + halo;
+    const int vcol = ctid & 15, rgrp = ctid >> 4, lane = ctid & 31;
+
+    // tiles are requested in unit order: (load_s, load_t) just advances (thread 0 of the role)
+    int load_s = (int)(u0 / p.F), load_t = (int)(u0 % p.F) - halo;
+    auto issue = [&](int q) {
+        const int slot = q % kNBuf;
+        mbar_expect_tx(sm.full + slot, p.tile_bytes);
+        tma_load_2d(sm.tiles + (size_t)slot * p.tile_stride, tmap, load_s * kSliceBytes, load_t * p.f,
+                    sm.full + slot);
+        if (++load_t == p.F) { load_t = 0; ++load_s; }
+    };
+    if (ctid == 0)
+        for (int q = 0; q < kNBuf && q < Q; ++q) issue(q);
+
+    Walk w;
+    w.start(p, u0);
+    for (int q = 0; q < Q; ++q) {
+        const int slot = q % kNBuf;
+        const uint32_t phase = (uint32_t)((q / kNBuf) & 1);
+        const bool halo_tile = halo && q == 0;
+        // the 128 threads leave together: a thread that saw a failed wait tells the others here
+        bool bad = *sm.abort_flag != 0;
+        if (!bad && !halo_tile && !mbar_wait(sm.full + slot, phase)) {
+            *sm.abort_flag = 1;
+            bad = true;
+        }
+        if (column_any(bad)) return;
+        if (halo_tile) {
+            if (lane == 0) mbar_arrive(sm.empty + slot);        // the column warps do not read the halo tile
         } else {
-            o[0] = pair_f32(v.x, v.y); o[H - 1] = pair_f32(v.z, v.w);
+            const int n = q - halo;
+            const unsigned char* tile = sm.tiles + (size_t)slot * p.tile_stride + vcol * 16;
+            f32x2 acc[H];
+#pragma unroll
+            for (int i = 0; i < H; ++i) acc[i] = pk(0.f, 0.f);
+            int r = rgrp;
+            for (; r + 3 * kColGroups < p.f; r += 4 * kColGroups) {
+                uint4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    v[u] = *reinterpret_cast<const uint4*>(tile + (r + u * kColGroups) * kSliceBytes);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    f32x2 a2[H];
+                    widen_pairs<DT>(v[u], a2);
+#pragma unroll
+                    for (int i = 0; i < H; ++i) acc[i] = add2(acc[i], a2[i]);
+                }
+            }
+            for (; r < p.f; r += kColGroups) {
+                f32x2 a2[H];
+                widen_pairs<DT>(*reinterpret_cast<const uint4*>(tile + r * kSliceBytes), a2);
+#pragma unroll
+                for (int i = 0; i < H; ++i) acc[i] = add2(acc[i], a2[i]);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sm.empty + slot);        // this warp is done with the tile
+            float* dst = sm.cs + rgrp * SE + vcol * P;
+#pragma unroll
+            for (int i = 0; i < H; i += 2)
+                *reinterpret_cast<ulonglong2*>(dst + 2 * i) = make_ulonglong2(acc[i], acc[i + 1]);
+            asm volatile("bar.sync 1, %0;" ::"n"(kColThreads) : "memory");
+            if (ctid < SE) {
+                float sum = 0.f;
+#pragma unroll
+                for (int gidx = 0; gidx < kColGroups; ++gidx) sum += sm.cs[gidx * SE + ctid];
+                const float m = sum / (float)p.f;
+                // the buffer was last used two tiles ago: wait until every row warp has read it
+                if (n >= 2 && !mbar_wait(sm.mean_empty + (n & 1), (uint32_t)(((n >> 1) + 1) & 1))) *sm.abort_flag = 1;
+                sm.mean_s[(n & 1) * SE + ctid] = m;
+                p.mean[(int64_t)w.t * p.d + w.s * SE + ctid] = m;
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(kColThreads) : "memory");
+            if (ctid == 0) mbar_arrive(sm.mean_full + (n & 1));
+            w.step(p);
+        }
+        // refill the buffer of the tile in front of this one as soon as every warp has let go of it
+        if (ctid == 0 && q >= 1 && q - 1 + kNBuf < Q) {
+            if (mbar_wait(sm.empty + ((q - 1) % kNBuf), (uint32_t)(((q - 1) / kNBuf) & 1))) issue(q - 1 + kNBuf);
+            else *sm.abort_flag = 1;                            // everyone leaves at the next check
         }
     }
+}
+
+// ---------------------------------------------------------------------------------------
+// row warps
+// ---------------------------------------------------------------------------------------
+template <int DT>
+struct RowState {
+    static constexpr int H = Elem<DT>::kPerVec / 2;
+    uint4 prev[kRows][2];   // previous frame's rows of this thread (two vectors each)
+    float bb[kRows];        // this thread's share of ||previous row||^2
+    int warp, g, j, f;
 
     // Row slot r of this thread is row 64 r + 4 warp + g (g = lane group): a warp owns four
     // consecutive rows per slot.  A slot is visited when its first row exists (a warp-uniform test);
     // lane groups whose row lies beyond the frame read the zero rows that pad every tile buffer to a
     // multiple of four rows, so no lane ever branches on its own row.
-    __device__ __forceinline__ bool slot_live(int r) const { return 64 * r + 4 * warp < p->f; }
+    __device__ __forceinline__ bool slot_live(int r) const { return 64 * r + 4 * warp < f; }
     __device__ __forceinline__ int slot_row(int r) const { return 64 * r + 4 * warp + g; }
     __device__ __forceinline__ const unsigned char* my_rows(const unsigned char* tile) const {
         return tile + (4 * warp + g) * kSliceBytes + j * 16;
     }
 
-    // Frame in front of the first unit: registers only.
+    // frame in front of the first unit: registers only
     __device__ __forceinline__ void load_halo(const unsigned char* tile) {
         const unsigned char* base = my_rows(tile);
 #pragma unroll
@@ -224,7 +375,7 @@ struct Pass {
                 for (int h = 0; h < 2; ++h) {
                     prev[r][h] = *reinterpret_cast<const uint4*>(base + r * (64 * kSliceBytes) + h * 128);
                     f32x2 b2[H];
-                    to_pairs(prev[r][h], b2);
+                    widen_pairs<DT>(prev[r][h], b2);
 #pragma unroll
                     for (int i = 0; i < H; ++i) acc = fma2(b2[i], b2[i], acc);
                 }
@@ -233,37 +384,10 @@ struct Pass {
         }
     }
 
-    // x[4r + 3] = <previous row, previous mean> over this thread's columns (the other entries 0),
-    // reduced over the row's 8 lanes and written to the previous frame's partial record.
-    __device__ __forceinline__ void flush_prev(int s, int t_prev) {
-        float x[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) x[i] = 0.f;
-#pragma unroll
-        for (int r = 0; r < kRows; ++r) {
-            if (slot_live(r)) {
-                f32x2 acc = pk(0.f, 0.f);
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    f32x2 b2[H];
-                    to_pairs(prev[r][h], b2);
-#pragma unroll
-                    for (int i = 0; i < H; ++i) acc = fma2(b2[i], mprev[h][i], acc);
-                }
-                x[4 * r + 3] = hsum(acc);
-            }
-        }
-        group8_reduce_scatter(x, j);
-        const int row = slot_row(j >> 1);
-        if ((j & 1) && row < p->f) p->part[((int64_t)t_prev * p->nsl + s) * p->f + row].w = x[1];
-    }
-
-    // Slots [R0, R1) of one tile, without a branch: everything the frame contributes per row.
-    //   HAS_PREV  the registers hold frame t-1 of this slice
-    //   TEMPORAL  ... and frame t continues the same video, so ||a-b||^2 is wanted
-    //   OWN_PREV  ... and frame t-1 was a unit of this CTA, so its <row, mean> is computed here
-    template <int R0, int R1, bool HAS_PREV, bool TEMPORAL, bool OWN_PREV>
-    __device__ __forceinline__ void slots(const unsigned char* base, f32x2 (&colsum)[2][H], float (&x)[16]) {
+    // slots [R0, R1) of one tile, without a branch: ||a||^2, ||a - m||^2 and, when the frame continues
+    // a video (TEMPORAL), ||a - b||^2 against the rows in registers, which the new rows then replace
+    template <int R0, int R1, bool TEMPORAL>
+    __device__ __forceinline__ void slots(const unsigned char* base, const f32x2 (&m)[2][H], float (&x)[16]) {
         uint4 a4[R1 - R0][2];
 #pragma unroll
         for (int r = R0; r < R1; ++r)
@@ -272,135 +396,123 @@ struct Pass {
                 a4[r - R0][h] = *reinterpret_cast<const uint4*>(base + r * (64 * kSliceBytes) + h * 128);
 #pragma unroll
         for (int r = R0; r < R1; ++r) {
-            f32x2 aa = pk(0.f, 0.f), db = aa, bm = aa;
+            f32x2 aa = pk(0.f, 0.f), dm = aa, db = aa;
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 f32x2 a2[H];
-                to_pairs(a4[r - R0][h], a2);
+                widen_pairs<DT>(a4[r - R0][h], a2);
 #pragma unroll
                 for (int i = 0; i < H; ++i) {
-                    colsum[h][i] = add2(colsum[h][i], a2[i]);
+                    const f32x2 e = sub2(a2[i], m[h][i]);
                     aa = fma2(a2[i], a2[i], aa);
+                    dm = fma2(e, e, dm);
                 }
-                if (HAS_PREV && (TEMPORAL || OWN_PREV)) {
+                if (TEMPORAL) {
                     f32x2 b2[H];
-                    to_pairs(prev[r][h], b2);
+                    widen_pairs<DT>(prev[r][h], b2);
 #pragma unroll
                     for (int i = 0; i < H; ++i) {
-                        if (TEMPORAL) {
-                            const f32x2 e = sub2(a2[i], b2[i]);
-                            db = fma2(e, e, db);
-                        }
-                        if (OWN_PREV) bm = fma2(b2[i], mprev[h][i], bm);
+                        const f32x2 e = sub2(a2[i], b2[i]);
+                        db = fma2(e, e, db);
                     }
                 }
                 prev[r][h] = a4[r - R0][h];
             }
             x[4 * r + 0] = hsum(aa);
-            x[4 * r + 1] = hsum(db);
-            x[4 * r + 2] = HAS_PREV ? bb[r] : 0.f;
-            x[4 * r + 3] = hsum(bm);
+            x[4 * r + 1] = hsum(dm);
+            x[4 * r + 2] = hsum(db);
+            x[4 * r + 3] = TEMPORAL ? bb[r] : 0.f;
             bb[r] = x[4 * r + 0];
         }
     }
 
-    // One unit: the tile of (slice s, frame t) in buffer `slot`; q is its place in the load order.
-    // Returns false when the CTA must stop (a bounded wait ran out).
-    template <bool HAS_PREV, bool TEMPORAL, bool OWN_PREV>
-    __device__ __forceinline__ bool unit(int q, int slot, uint32_t phase, int s, int t) {
-        const FusedParams& pp = *p;
-        const unsigned char* base = my_rows(wait_tile(slot, phase));
-
-        f32x2 colsum[2][H];
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int i = 0; i < H; ++i) colsum[h][i] = pk(0.f, 0.f);
-        float x[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) x[i] = 0.f;
+    template <bool TEMPORAL>
+    __device__ __forceinline__ void tile_pass(const unsigned char* tile, const f32x2 (&m)[2][H], float (&x)[16]) {
+        const unsigned char* base = my_rows(tile);
         if (slot_live(2)) {                     // the usual case: a straight run over three slots
-            slots<0, 2, HAS_PREV, TEMPORAL, OWN_PREV>(base, colsum, x);
-            slots<2, 3, HAS_PREV, TEMPORAL, OWN_PREV>(base, colsum, x);
-            if (slot_live(3)) slots<3, 4, HAS_PREV, TEMPORAL, OWN_PREV>(base, colsum, x);
+            slots<0, 2, TEMPORAL>(base, m, x);
+            slots<2, 3, TEMPORAL>(base, m, x);
+            if (slot_live(3)) slots<3, 4, TEMPORAL>(base, m, x);
         } else {
-            if (slot_live(0)) slots<0, 1, HAS_PREV, TEMPORAL, OWN_PREV>(base, colsum, x);
-            if (slot_live(1)) slots<1, 2, HAS_PREV, TEMPORAL, OWN_PREV>(base, colsum, x);
+            if (slot_live(0)) slots<0, 1, TEMPORAL>(base, m, x);
+            if (slot_live(1)) slots<1, 2, TEMPORAL>(base, m, x);
         }
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            float* dst = cs + rgid * SE + (j + 8 * h) * P;
-#pragma unroll
-            for (int i = 0; i < H; i += 2)
-                *reinterpret_cast<ulonglong2*>(dst + 2 * i) = make_ulonglong2(colsum[h][i], colsum[h][i + 1]);
-        }
-        __syncthreads();                            // tile buffer free, column partials visible
-        if (*abort_flag) return false;
-        if (tid == 0 && q + pp.nbuf < Q) issue_load(q + pp.nbuf);
-        // column sums over the 64 row groups: fixed order, two levels
-#pragma unroll
-        for (int e = tid; e < 4 * SE; e += kThreads) {
-            const int col = e % SE, quarter = e / SE;
-            float sum = 0.f;
-#pragma unroll
-            for (int i = 0; i < kRowGroups / 4; ++i) sum += cs[(quarter * (kRowGroups / 4) + i) * SE + col];
-            cs2[quarter * SE + col] = sum;
-        }
-
-        // per-row partial sums of the slice (overlaps the mean reduction of the other warps)
-        group8_reduce_scatter(x, j);
-        {
-            const int row = slot_row(j >> 1);
-            if (row < pp.f) {
-                float4* rec = pp.part + ((int64_t)t * pp.nsl + s) * pp.f + row;
-                if (j & 1) {
-                    rec->z = x[0];                                              // ||b||^2
-                    if (OWN_PREV) (rec - (int64_t)pp.nsl * pp.f)->w = x[1];     // frame t-1: <b, mean>
-                } else {
-                    *reinterpret_cast<float2*>(rec) = make_float2(x[0], x[1]);  // ||a||^2, ||a-b||^2
-                }
-            }
-        }
-        __syncthreads();
-        if (tid < SE) {
-            const float m = ((cs2[tid] + cs2[SE + tid]) + (cs2[2 * SE + tid] + cs2[3 * SE + tid])) / (float)pp.f;
-            mean_s[tid] = m;
-            pp.mean[(int64_t)t * pp.d + s * SE + tid] = m;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int i = 0; i < H; ++i)
-                mprev[h][i] = *reinterpret_cast<const f32x2*>(mean_s + (j + 8 * h) * P + 2 * i);
-        return true;
-    }
-
-    __device__ __forceinline__ bool unit_dispatch(int q, int slot, uint32_t phase, int s, int t, bool has_prev,
-                                                  bool own_prev, bool is_first) {
-        if (!has_prev) return unit<false, false, false>(q, slot, phase, s, t);
-        if (!is_first)
-            return own_prev ? unit<true, true, true>(q, slot, phase, s, t)
-                            : unit<true, true, false>(q, slot, phase, s, t);
-        return own_prev ? unit<true, false, true>(q, slot, phase, s, t)
-                        : unit<true, false, false>(q, slot, phase, s, t);
     }
 };
 
 template <int DT>
+__device__ __forceinline__ void row_role(const FusedParams& p, Smem<DT>& sm, int64_t u0, int n_units, int halo,
+                                         int tid) {
+    using E = Elem<DT>;
+    constexpr int P = E::kPerVec, H = P / 2, SE = Smem<DT>::SE;
+    const int lane = tid & 31;
+    RowState<DT> st;
+    st.warp = tid >> 5;
+    st.g = lane >> 3;
+    st.j = lane & 7;
+    st.f = p.f;
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) {
+        st.prev[r][0] = make_uint4(0u, 0u, 0u, 0u);
+        st.prev[r][1] = st.prev[r][0];
+        st.bb[r] = 0.f;
+    }
+    int q = 0;
+    bool has_prev = false;
+    if (halo) {
+        if (!__all_sync(0xffffffffu, mbar_wait(sm.full + 0, 0))) { *sm.abort_flag = 1; return; }
+        st.load_halo(sm.tiles);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sm.empty + 0);
+        q = 1;
+        has_prev = true;
+    }
+    Walk w;
+    w.start(p, u0);
+    for (int n = 0; n < n_units; ++n, ++q) {
+        const int slot = q % kNBuf;
+        // a warp leaves as a whole: the lanes agree on what they saw
+        const bool fine = *sm.abort_flag == 0 && mbar_wait(sm.full + slot, (uint32_t)((q / kNBuf) & 1)) &&
+                          mbar_wait(sm.mean_full + (n & 1), (uint32_t)((n >> 1) & 1));
+        if (!__all_sync(0xffffffffu, fine)) {
+            *sm.abort_flag = 1;
+            return;
+        }
+        f32x2 m[2][H];
+        const float* ms = sm.mean_s + (n & 1) * SE;
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int i = 0; i < H; ++i)
+                m[h][i] = *reinterpret_cast<const f32x2*>(ms + (st.j + 8 * h) * P + 2 * i);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sm.mean_empty + (n & 1));
+
+        float x[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) x[i] = 0.f;
+        const unsigned char* tile = sm.tiles + (size_t)slot * p.tile_stride;
+        if (has_prev && !w.is_first) st.template tile_pass<true>(tile, m, x);
+        else st.template tile_pass<false>(tile, m, x);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sm.empty + slot);            // this warp is done with the tile
+
+        // per-row sums of the slice: reduce over the row's 8 lanes, one record per row
+        group8_reduce_scatter(x, st.j);
+        const int row = st.slot_row(st.j >> 1);
+        if (row < p.f) {
+            float2* rec = reinterpret_cast<float2*>(p.part + ((int64_t)w.t * p.nsl + w.s) * p.f + row);
+            rec[st.j & 1] = make_float2(x[0], x[1]);    // even lane: ||a||^2, ||a-m||^2; odd: ||a-b||^2, ||b||^2
+        }
+        has_prev = !w.step(p);                          // a new slice starts without a previous frame
+    }
+}
+
+template <int DT>
 __global__ void __launch_bounds__(kThreads, 1)
 score_pass_kernel(const __grid_constant__ CUtensorMap tmap, const FusedParams p, int32_t* status_word) {
-    constexpr int SE = Pass<DT>::SE;
     extern __shared__ __align__(1024) unsigned char smem[];
-    Pass<DT> c;
-    c.tmap = &tmap;
-    c.p = &p;
-    c.tiles = smem;
-    c.cs = reinterpret_cast<float*>(smem + (size_t)p.nbuf * p.tile_stride);
-    c.cs2 = c.cs + kRowGroups * SE;
-    c.mean_s = c.cs2 + 4 * SE;
-    c.bars = reinterpret_cast<uint64_t*>(c.mean_s + SE);
-    c.abort_flag = reinterpret_cast<volatile int*>(c.bars + 4);
+    Smem<DT> sm(smem, p.tile_stride);
 
     // let the finaliser's CTAs be scheduled as soon as SMs free up; they wait for this whole grid
     cudaTriggerProgrammaticLaunchCompletion();
@@ -409,104 +521,53 @@ score_pass_kernel(const __grid_constant__ CUtensorMap tmap, const FusedParams p,
     const int64_t u0 = U * blockIdx.x / gridDim.x;
     const int64_t u1 = U * (blockIdx.x + 1) / gridDim.x;
     if (u0 >= u1) return;
-    int s = (int)(u0 / p.F), t = (int)(u0 % p.F);
+    const int n_units = (int)(u1 - u0);
+    const int t0 = (int)(u0 % p.F);
+    const int vid0 = upper_segment(p.video_frame_offsets, p.num_videos, t0);
+    const int halo = (__ldg(p.video_frame_offsets + vid0) == t0) ? 0 : 1;
 
-    // videos: `vid` is the video of frame t, `next_start` the first frame of the next one
-    int vid = upper_segment(p.video_frame_offsets, p.num_videos, t);
-    bool is_first = __ldg(p.video_frame_offsets + vid) == t;
-    int next_start = __ldg(p.video_frame_offsets + vid + 1);
-
-    c.halo = is_first ? 0 : 1;
-    c.Q = (int)(u1 - u0) + c.halo;
-    c.load_s = s;
-    c.load_t = t - c.halo;
-
-    const int tid = threadIdx.x, lane = tid & 31;
-    c.tid = tid;
-    c.warp = tid >> 5;
-    c.g = lane >> 3;
-    c.j = lane & 7;
-    c.rgid = c.warp * 4 + c.g;
+    const int tid = threadIdx.x;
     if (tid == 0) {
-        for (int i = 0; i < p.nbuf; ++i) mbar_init(c.bars + i, 1);
-        *c.abort_flag = 0;
+        for (int i = 0; i < kNBuf; ++i) {
+            mbar_init(sm.full + i, 1);
+            mbar_init(sm.empty + i, kRowWarps + kColWarps);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(sm.mean_full + i, 1);
+            mbar_init(sm.mean_empty + i, kRowWarps);
+        }
+        *sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     // rows beyond the frame in every tile buffer stay zero for the whole kernel (TMA writes f rows)
-    for (int b = 0; b < p.nbuf; ++b) {
-        uint4* pad = reinterpret_cast<uint4*>(c.tiles + (size_t)b * p.tile_stride + p.tile_bytes);
+    for (int b = 0; b < kNBuf; ++b) {
+        uint4* pad = reinterpret_cast<uint4*>(sm.tiles + (size_t)b * p.tile_stride + p.tile_bytes);
         const int n = (int)((p.tile_stride - p.tile_bytes) / 16);
         for (int i = tid; i < n; i += kThreads) pad[i] = make_uint4(0u, 0u, 0u, 0u);
     }
     __syncthreads();
-    if (tid == 0)
-        for (int q = 0; q < p.nbuf && q < c.Q; ++q) c.issue_load(q);
 
-#pragma unroll
-    for (int r = 0; r < kRows; ++r) {
-        c.prev[r][0] = make_uint4(0u, 0u, 0u, 0u);
-        c.prev[r][1] = c.prev[r][0];
-        c.bb[r] = 0.f;
-    }
-
-    int q = 0, slot = 0;
-    uint32_t phase = 0;
-    bool ok = true, has_prev = false, own_prev = false;
-    if (c.halo) {
-        c.load_halo(c.wait_tile(0, 0));
-        __syncthreads();
-        ok = *c.abort_flag == 0;
-        if (ok && tid == 0 && p.nbuf < c.Q) c.issue_load(p.nbuf);
-        q = 1;
-        if (++slot == p.nbuf) { slot = 0; phase ^= 1; }
-        has_prev = true;
-    }
-    const int n_units = (int)(u1 - u0);
-    for (int i = 0; ok && i < n_units; ++i) {
-        ok = c.unit_dispatch(q, slot, phase, s, t, has_prev, own_prev, is_first);
-        has_prev = true;
-        own_prev = true;
-        ++q;
-        if (++slot == p.nbuf) { slot = 0; phase ^= 1; }
-        // next unit
-        if (++t == p.F) {                           // the range crosses into the next slice
-            if (ok) c.flush_prev(s, p.F - 1);
-            t = 0;
-            ++s;
-            has_prev = false;
-            own_prev = false;
-            vid = upper_segment(p.video_frame_offsets, p.num_videos, 0);
-            next_start = __ldg(p.video_frame_offsets + vid + 1);
-            is_first = true;
-        } else {
-            is_first = false;
-            while (t >= next_start && vid + 1 < p.num_videos) {     // skips videos without frames
-                ++vid;
-                is_first = true;
-                next_start = __ldg(p.video_frame_offsets + vid + 1);
-            }
-        }
-    }
-    if (ok) {
-        if (own_prev) c.flush_prev((int)((u1 - 1) / p.F), (int)((u1 - 1) % p.F));
+    // The block is launched with 96 registers per thread (640 x 96 = 61440).  The column warps give
+    // most of theirs back and the four row warpgroups take 8 more each: 128 x 48 + 512 x 104 = 59392.
+    if (tid < kRowThreads) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 104;");
+        row_role<DT>(p, sm, u0, n_units, halo, tid);
     } else {
-        // A wait on the CTA's own loads ran out.  Report it, then give the loads that are still in
-        // flight one more bounded wait each, so that nothing lands in shared memory after exit.
-        __syncthreads();
-        if (tid == 0) {
-            report(status_word, SHARPV_ERR_TIMEOUT);
-            const int last = min(c.Q, q + p.nbuf);
-            for (int i = q; i < last; ++i) (void)mbar_wait(c.bars + (i % p.nbuf), (uint32_t)((i / p.nbuf) & 1));
-        }
-        __syncthreads();
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+        column_role<DT>(&tmap, p, sm, u0, n_units, halo, tid - kRowThreads);
     }
-}
 
-// ||a^ - b^||^2 from <a,a>, <b,b>, <a,b>; a zero vector normalises to zero
-__device__ __forceinline__ float dissim_sq_from_dot(float saa, float sbb, float sab) {
-    const float ca = fmaxf(sqrtf(saa), kNormEps), cb = fmaxf(sqrtf(sbb), kNormEps);
-    return fmaxf(saa / (ca * ca) + sbb / (cb * cb) - 2.f * sab / (ca * cb), 0.f);
+    __syncthreads();
+    if (*sm.abort_flag && tid == 0) {
+        // A bounded wait ran out.  Report it, then give every tile buffer one more bounded wait so
+        // that no load lands in shared memory after the CTA has gone.
+        report(status_word, SHARPV_ERR_TIMEOUT);
+        for (int i = 0; i < kNBuf; ++i) {
+            (void)mbar_wait(sm.full + i, 0);
+            (void)mbar_wait(sm.full + i, 1);
+        }
+    }
 }
 
 // One CTA per frame: adds the slices in a fixed order, writes S, T, I, ratio_t and k_t.
@@ -557,12 +618,12 @@ score_finalize_kernel(const FusedParams p) {
 
     if (tid < p.f) {
         const float4 a0 = g_sum[0][tid], a1 = g_sum[1][tid], a2 = g_sum[2][tid], a3 = g_sum[3][tid];
-        const float aa = (a0.x + a1.x) + (a2.x + a3.x), db = (a0.y + a1.y) + (a2.y + a3.y);
-        const float bb = (a0.z + a1.z) + (a2.z + a3.z), am = (a0.w + a1.w) + (a2.w + a3.w);
-        const float s2 = dissim_sq_from_dot(aa, smm, am);
+        const float aa = (a0.x + a1.x) + (a2.x + a3.x), dm = (a0.y + a1.y) + (a2.y + a3.y);
+        const float db = (a0.z + a1.z) + (a2.z + a3.z), bb = (a0.w + a1.w) + (a2.w + a3.w);
+        const float s2 = dissim_sq_from_sums(aa, smm, dm);
         const float t2 = is_first ? 0.f : dissim_sq_from_sums(aa, bb, db);
         int fl = 0;
-        if (s2 < kRefineBelow) fl |= 1;
+        if (s2 < kRefineBelow && dm != 0.f) fl |= 1;
         if (!is_first && t2 < kRefineBelow && db != 0.f) fl |= 2;
         f_s2[tid] = s2; f_t2[tid] = t2; f_aa[tid] = aa; f_bb[tid] = bb; f_fl[tid] = fl;
     }
@@ -608,8 +669,6 @@ score_finalize_kernel(const FusedParams p) {
     }
 }
 
-size_t fixed_smem_bytes(int se) { return (size_t)(kRowGroups * se + 4 * se + se) * 4 + 4 * 8 + 16; }
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -630,10 +689,7 @@ EncodeTiledFn encode_fn() {
 
 template <int DT>
 sharpv_status launch(const FusedScoreArgs& a, const CUtensorMap& tmap, FusedParams& p, int sms) {
-    const size_t fixed = fixed_smem_bytes(Pass<DT>::SE);
-    p.nbuf = 3;
-    while (p.nbuf > 1 && (size_t)p.nbuf * p.tile_stride + fixed > (size_t)kSmemBudget) --p.nbuf;
-    const size_t smem = (size_t)p.nbuf * p.tile_stride + fixed;
+    const size_t smem = (size_t)kNBuf * p.tile_stride + Smem<DT>::fixed_bytes();
     if (smem > (size_t)kSmemBudget) return SHARPV_ERR_UNSUPPORTED;
     if (cudaFuncSetAttribute(score_pass_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess) {
@@ -679,7 +735,6 @@ sharpv_status fused_score_launch(const FusedScoreArgs& a) {
     p.F = a.F; p.f = a.f; p.d = a.d;
     p.nsl = (int)((int64_t)a.d * eb / kSliceBytes);
     p.nvec = a.d * eb / 16;
-    p.nbuf = 3;
     p.num_videos = a.num_videos;
     p.video_frame_offsets = a.video_frame_offsets;
     p.w = a.w; p.one_minus_cos = a.one_minus_cos; p.round_mode = a.round_mode; p.min_keep = a.min_keep;
