@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--stage", default=None, choices=["score", "select", "calibrate", "compact"],
                     help="profiling aid: after the warm-up run only this entry point --steps times "
                          "(L2 flushed before each) and print its mean duration")
+    ap.add_argument("--inplace", action="store_true",
+                    help="compact the K/V cache in place (kv_dst == kv_src) instead of into a second cache")
     ap.add_argument("--layers", type=int, default=None,
                     help="override the number of K/V layers (profiling aid: smaller device footprint)")
     ap.add_argument("--frames", type=int, default=None,
@@ -302,8 +304,8 @@ def run_sharpv(args):
                                      capacity=T, out=o_cal, workspace=ws_cal, status_word=status)
 
     def stage_compact(i=0):
-        sv.sharpv_kv_compact(kv, kv_dst, o_cal["kept_pos"], o_cal["kept_seq_offsets"], capacity=T,
-                             status_word=status)
+        sv.sharpv_kv_compact(kv, kv if args.inplace else kv_dst, o_cal["kept_pos"], o_cal["kept_seq_offsets"],
+                             capacity=T, status_word=status)
 
     stages = [("score", stage_score), ("select", stage_select), ("calibrate", stage_calibrate),
               ("compact", stage_compact)]
@@ -463,7 +465,7 @@ def run_sharpv(args):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "frames": F, "tokens_per_frame": f, "d": d, "storage": wl.dtype,
                    "visual_tokens": NV, "seq_tokens": T, "kv": list(wl.kv_shape()), "M": args.M, "w": args.w,
-                   "kept_stage_one": n_keep, "kept_stage_two": t_keep,
+                   "kept_stage_one": n_keep, "kept_stage_two": t_keep, "kv_in_place": bool(args.inplace),
                    "launch": "one CUDA graph replay per step, steps back to back",
                    "l2": "inputs larger than L2: a step streams several times the 126 MB L2 (K/V alone is "
                          "larger), and the per-kernel timings rotate through input copies totalling more than "

@@ -213,7 +213,9 @@ sharpv_status sharpv_kv_calibrate_prune_noalloc(
  * as a bit copy of head_dim elements.  Strides are in elements; the head_dim axis is
  * contiguous; every stride * sizeof(element) and head_dim * sizeof(element) must be a
  * multiple of 16 bytes.  The benchmarked layout is [L][2][H][T][D_h]; a token-major cache is
- * expressed through the strides.  dst must not overlap src.  Rows of dst at and beyond
+ * expressed through the strides.  kv_dst == kv_src with identical strides compacts in place (every
+ * plane is walked front to back; serving stacks that cannot afford a second cache use this);
+ * otherwise dst must not overlap src.  Rows of dst at and beyond
  * n_kept are left untouched.  `capacity` is an upper bound on n_kept that the host knows
  * (for example total_seq_tokens) and sizes the launch; rows beyond it are not copied.
  */

@@ -308,3 +308,30 @@ void sharpv_oracle_kv_compact(const void *src, void *dst, int num_kv_heads, int6
             memcpy(o + j * dst_stride_token, s + (int64_t)kept_pos[j] * src_stride_token, (size_t)row_bytes);
     }
 }
+
+/*
+ * In-place variant of the K/V compaction: within every plane, row j becomes the old row kept_pos[j]
+ * for j < n_kept, everything behind stays as it was.  Written as "copy the plane, then gather from
+ * the copy", which is the definition and cannot alias.
+ */
+int sharpv_oracle_kv_compact_inplace(void *kv, int num_kv_heads, int64_t row_bytes,
+                                     int64_t stride_layer, int64_t stride_kv, int64_t stride_head,
+                                     int64_t stride_token, int64_t tokens, int layer_begin, int layer_end,
+                                     const int32_t *kept_pos, int64_t n_kept)
+{
+    int planes = (layer_end - layer_begin) * 2 * num_kv_heads;
+    char *copy = (char *)malloc((size_t)(tokens > 0 ? tokens : 1) * (size_t)row_bytes);
+    if (!copy) return -1;
+    for (int p = 0; p < planes; ++p) {
+        int l = layer_begin + p / (2 * num_kv_heads);
+        int kv_i = (p / num_kv_heads) % 2;
+        int h = p % num_kv_heads;
+        char *base = (char *)kv + l * stride_layer + kv_i * stride_kv + h * stride_head;
+        for (int64_t t = 0; t < tokens; ++t)
+            memcpy(copy + t * row_bytes, base + t * stride_token, (size_t)row_bytes);
+        for (int64_t j = 0; j < n_kept; ++j)
+            memcpy(base + j * stride_token, copy + (int64_t)kept_pos[j] * row_bytes, (size_t)row_bytes);
+    }
+    free(copy);
+    return 0;
+}

@@ -184,3 +184,20 @@ def kv_compact(kv_src: np.ndarray, kept_pos, layer_begin: int = 0, layer_end: Op
         C.c_int64(ds[0]), C.c_int64(ds[1]), C.c_int64(ds[2]), C.c_int64(ds[3]),
         C.c_int(layer_begin), C.c_int(layer_end), _ptr(kp), C.c_int64(kp.size), C.c_int(nthreads))
     return dst
+
+
+def kv_compact_inplace(kv: np.ndarray, kept_pos, layer_begin: int = 0, layer_end: Optional[int] = None) -> np.ndarray:
+    """In-place compaction of kv [L, 2, H, T, D_h] (modifies and returns kv)."""
+    assert kv.ndim == 5 and kv.strides[4] == kv.itemsize
+    kp = np.ascontiguousarray(kept_pos, dtype=np.int32)
+    L, _, H, T, Dh = kv.shape
+    if layer_end is None:
+        layer_end = L
+    st = kv.strides
+    fn = lib().sharpv_oracle_kv_compact_inplace
+    fn.restype = C.c_int
+    rc = fn(_ptr(kv), C.c_int(H), C.c_int64(Dh * kv.itemsize), C.c_int64(st[0]), C.c_int64(st[1]), C.c_int64(st[2]),
+            C.c_int64(st[3]), C.c_int64(T), C.c_int(layer_begin), C.c_int(layer_end), _ptr(kp), C.c_int64(kp.size))
+    if rc != 0:
+        raise RuntimeError("sharpv_oracle_kv_compact_inplace failed")
+    return kv

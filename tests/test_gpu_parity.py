@@ -220,6 +220,69 @@ def test_kv_compact_layouts_and_layer_range():
     np.testing.assert_array_equal(to_host(dst_tm)[:, :, :kept.size], wl.kv[:, :, :, kept].transpose(0, 1, 3, 2, 4))
 
 
+@pytest.mark.parametrize("name", ["tiny", "small_ragged", "odd_shapes", "onevision_7b"])
+@pytest.mark.parametrize("M", [0.2, 0.788])
+def test_kv_compact_in_place(name, M):
+    """kv_dst == kv_src: the kept prefix of every plane equals the gathered rows, the tail keeps its old
+    contents, bit for bit (oracle: copy each plane, gather from the copy)."""
+    wl, dw = _case(name)
+    T = wl.total_seq_tokens
+    g = sv.sharpv_kv_calibrate_prune(dw.hidden, dw.tokens, dw.seq_offsets, dw.vis_begin, dw.vis_count,
+                                     dw.vis_offsets, T, M=M)
+    torch.cuda.synchronize()
+    n = int(g["kept_seq_offsets"][-1].item())
+    kept = to_host(g["kept_pos"])[:n]
+    kv = dw.kv.clone()
+    sv.sharpv_kv_compact(kv, kv, g["kept_pos"], g["kept_seq_offsets"], capacity=T)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(to_host(kv), orc.kv_compact_inplace(wl.kv.copy(), kept))
+    # token-major cache, layers [1, L) only
+    L = wl.num_layers
+    if L > 1:
+        tm = dw.kv.permute(0, 1, 3, 2, 4).contiguous()
+        view = tm.permute(0, 1, 3, 2, 4)
+        sv.sharpv_kv_compact(view, view, g["kept_pos"], g["kept_seq_offsets"], capacity=T, layer_begin=1)
+        torch.cuda.synchronize()
+        expect = np.ascontiguousarray(wl.kv.transpose(0, 1, 3, 2, 4))
+        orc.kv_compact_inplace(expect.transpose(0, 1, 3, 2, 4), kept, layer_begin=1)
+        np.testing.assert_array_equal(to_host(tm), expect)
+
+
+def test_layer_wise_reading_of_eq7():
+    """Eq. 7 read layer by layer (hierarchical cache pruning): every layer has its own hidden state, its own
+    kept set and compacts only its own K/V.  Built from the same two entry points, one call per layer."""
+    L = 4
+    wl = W.custom("layers", 90, W.BF16, 8, 512, 16, [W.make_video_spec(6, 0.9, cuts=[3])], 0.0, L, 2, 64)
+    W.fill_tokens(wl)
+    W.fill_kv(wl)
+    dw_tokens = to_dev(wl.tokens)
+    i32 = lambda a: torch.from_numpy(a).cuda()
+    tabs = [i32(wl.seq_offsets), i32(wl.vis_begin), i32(wl.vis_count), i32(wl.vis_offsets)]
+    T, M = wl.total_seq_tokens, 0.6
+    kv = to_dev(wl.kv)
+    expect = wl.kv.copy()
+    means, counts = [], []
+    for l in range(L):
+        W.fill_hidden(wl, s_max=0.5 + 1.0 * l)          # deeper layers drift further from the visual features
+        hid = to_dev(wl.hidden)
+        g = sv.sharpv_kv_calibrate_prune(hid, dw_tokens, *tabs, T, M=M, want_mean_cos=True)
+        sv.sharpv_kv_compact(kv, kv, g["kept_pos"], g["kept_seq_offsets"], capacity=T, layer_begin=l, layer_end=l + 1)
+        torch.cuda.synchronize()
+        o = orc.kv_calibrate_prune(wl.hidden, wl.tokens, wl.seq_offsets, wl.vis_begin, wl.vis_count,
+                                   wl.vis_offsets, M)
+        n = int(g["kept_seq_offsets"][-1].item())
+        kept = to_host(g["kept_pos"])[:n]
+        assert np.setxor1d(kept, o["kept_pos"]).size <= 2
+        orc.kv_compact_inplace(expect, kept, layer_begin=l, layer_end=l + 1)
+        means.append(float(g["mean_cos"][0].item()))
+        counts.append(n)
+        assert abs(means[-1] - o["cos"].mean()) <= 1e-5
+    np.testing.assert_array_equal(to_host(kv), expect)
+    assert all(a > b for a, b in zip(means, means[1:]))     # similarity decays with depth ...
+    assert all(a >= b for a, b in zip(counts, counts[1:]))  # ... and so does the kept cache
+    assert counts[0] > counts[-1] >= wl.n_text
+
+
 def test_capacity_overflow_is_reported_not_written():
     wl, dw = _case("tiny")
     F, f, T = wl.total_frames, wl.f, wl.total_seq_tokens

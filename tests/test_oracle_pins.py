@@ -394,6 +394,22 @@ def test_kv_compact_is_fancy_indexing():
     np.testing.assert_array_equal(out3, out)
 
 
+def test_kv_compact_inplace_equals_out_of_place_prefix():
+    rng = np.random.default_rng(35)
+    L, H, T, Dh = 2, 3, 41, 8
+    kv = rng.integers(0, 65536, (L, 2, H, T, Dh)).astype(np.uint16)
+    kept = np.array([0, 1, 2, 9, 10, 30, 39, 40], np.int32)       # a leading run that stays where it is
+    ref = kv.copy()
+    out = orc.kv_compact_inplace(kv.copy(), kept)
+    np.testing.assert_array_equal(out[:, :, :, :kept.size], ref[:, :, :, kept])     # fancy indexing
+    np.testing.assert_array_equal(out[:, :, :, kept.size:], ref[:, :, :, kept.size:])   # tail untouched
+    # a token-major cache and a layer range
+    tm = np.ascontiguousarray(ref.transpose(0, 1, 3, 2, 4))
+    orc.kv_compact_inplace(tm.transpose(0, 1, 3, 2, 4), kept, layer_begin=1, layer_end=2)
+    np.testing.assert_array_equal(tm[0], ref[0].transpose(0, 2, 1, 3))
+    np.testing.assert_array_equal(tm[1][:, :kept.size], ref[1][:, :, kept].transpose(0, 2, 1, 3))
+
+
 def test_multithreaded_oracle_is_identical():
     wl = W.fill_hidden(W.fill_tokens(W.custom("mt", 34, W.BF16, 4, 64, 5, [W.make_video_spec(6, 0.9, cuts=[3])])))
     a = orc.score_frames(wl.tokens, wl.video_frame_offsets, wl.f, nthreads=1)
