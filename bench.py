@@ -31,7 +31,7 @@ FALLBACK_HBM_GBS = 6650.0
 # kernels launched per step by each entry point (score, select, calibrate, compact)
 LAUNCHES_PER_STEP = {"score": 2, "select": 2, "calibrate": 2, "compact": 1}
 # DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/); None = not captured
-NCU_TRAFFIC_BYTES = {("onevision_7b", "compact"): 267_609_600}   # profiles/kv_compact_kernel_onevision_7b.md
+NCU_TRAFFIC_BYTES = {("onevision_7b", "compact"): 266_712_320}   # profiles/kv_compact_kernel_onevision_7b.md
 
 
 def parse_args():
