@@ -4,9 +4,10 @@
 //
 // Kernels:
 //   count_above_kernel   (threshold variant only) per-frame count of I > K
-//   select_frame_kernel  one CTA per frame: its offset (sum of the budgets in front of it), a radix
-//                        select of the k-th largest key in shared memory, then an index-ordered
-//                        scan that writes ascending indices
+//   select_frame_kernel  one CTA per frame: its offset (sum of the budgets in front of it), then in
+//                        shared memory either a rank count over composite (key, index) keys (frames
+//                        of up to 1024 tokens) or a 4-pass byte radix select of the k-th largest key
+//                        with an index-ordered scan for the tie-break; ascending indices out
 //   gather_rows_kernel   one warp per kept row, 128-bit copies; launched as a dependent of the
 //                        selection so that its start-up overlaps it
 #include "common.cuh"
@@ -16,6 +17,7 @@ namespace {
 
 constexpr int kSelectThreads = 256;
 constexpr int kMaxTokensPerFrame = 8192;
+constexpr int kRankMaxTokens = 1024;     // frames up to this size are selected by counting ranks
 
 // Monotone map fp32 -> uint32: larger score, larger key.  Adding +0 turns -0 into +0.
 __device__ __forceinline__ uint32_t order_key(float x) {
@@ -44,7 +46,7 @@ __global__ void __launch_bounds__(kSelectThreads)
 select_frame_kernel(const float* __restrict__ importance, const int32_t* __restrict__ k, int F, int f,
                     int64_t capacity, int mode, float K, int32_t* __restrict__ kept_offsets,
                     int32_t* __restrict__ num_kept, int32_t* __restrict__ out_kept_index, int32_t* status_word) {
-    extern __shared__ uint32_t keys[];                 // [f]
+    extern __shared__ __align__(16) uint32_t keys[];   // [f]
     __shared__ int hist[4][256];                       // one histogram per byte pass, cleared once
     __shared__ int scan_sm[kSelectThreads / 32 + 1];
     __shared__ int off_sm[kSelectThreads / 32];
@@ -85,6 +87,36 @@ select_frame_kernel(const float* __restrict__ importance, const int32_t* __restr
         const int kt = min(max(kt_raw, 0), f);
         if (kt == 0) return;
         keep_all = kt == f;
+        if (!keep_all && f <= kRankMaxTokens) {
+            // Small frames: a token's rank under (key descending, index ascending) is the number of
+            // composite keys (key, ~index) above its own; it is kept iff rank < k.  No histogram,
+            // no pass structure: one sweep over shared memory, then one scan for the positions.
+            unsigned long long* comp = reinterpret_cast<unsigned long long*>(keys + ((f + 3) & ~3));
+            const int fpad = (f + 1) & ~1;
+            for (int i = tid; i < fpad; i += kSelectThreads)
+                comp[i] = i < f ? (((unsigned long long)keys[i] << 32) | (0xffffffffu - (uint32_t)i)) : 0ull;
+            __syncthreads();
+            int carry = 0;
+            for (int base = 0; base < f; base += kSelectThreads) {
+                const int i = base + tid;
+                const bool valid = i < f;
+                const unsigned long long mine = valid ? comp[i] : ~0ull;
+                int rank = 0;
+                for (int j = 0; j < fpad; j += 2) {
+                    const ulonglong2 c = *reinterpret_cast<const ulonglong2*>(comp + j);
+                    rank += (c.x > mine) + (c.y > mine);
+                }
+                const bool keep = valid && rank < kt;
+                int total;
+                const int pos = carry + block_exclusive_scan<kSelectThreads>(keep ? 1 : 0, scan_sm, total);
+                carry += total;
+                if (keep) {
+                    const int64_t j = out_base + pos;
+                    if (j < capacity) out_kept_index[j] = t * f + i;
+                }
+            }
+            return;
+        }
         if (!keep_all) {
             // radix select, most significant byte first: after the four passes `prefix` is the
             // k-th largest key and `remaining` says how many keys equal to it are still owed
@@ -211,7 +243,9 @@ sharpv_status select_impl(int mode, const float* importance, const int32_t* k, f
             return SHARPV_ERR_CUDA;
         return SHARPV_OK;
     }
-    if (launch_dependent(select_frame_kernel, dim3((unsigned)F), dim3(kSelectThreads), (size_t)f * 4, stream,
+    // keys, plus the 64-bit composite keys of the rank-counting path for small frames
+    const size_t sel_smem = (size_t)((f + 3) & ~3) * 4 + (f <= kRankMaxTokens ? (size_t)((f + 1) & ~1) * 8 : 0);
+    if (launch_dependent(select_frame_kernel, dim3((unsigned)F), dim3(kSelectThreads), sel_smem, stream,
                          importance, budgets, (int)F, (int)f, capacity, mode, K, out_kept_offsets, out_num_kept,
                          out_kept_index, status_word) != cudaSuccess) {
         (void)cudaGetLastError();
