@@ -264,8 +264,7 @@ __device__ __forceinline__ void column_role(const CUtensorMap* tmap, const Fused
 
     // tiles are requested in unit order: (load_s, load_t) just advances (thread 0 of the role)
     int load_s = (int)(u0 / p.F), load_t = (int)(u0 % p.F) - halo;
-    auto issue = [&](int q) {
-        const int slot = q % kNBuf;
+    auto issue = [&](int slot) {
         mbar_expect_tx(sm.full + slot, p.tile_bytes);
         tma_load_2d(sm.tiles + (size_t)slot * p.tile_stride, tmap, load_s * kSliceBytes, load_t * p.f,
                     sm.full + slot);
@@ -276,9 +275,11 @@ __device__ __forceinline__ void column_role(const CUtensorMap* tmap, const Fused
 
     Walk w;
     w.start(p, u0);
+    // ring position of tile q and of tile q-1, and the mean buffer of unit n, all kept incrementally
+    int slot = 0, prev_slot = 0, mb = 0;
+    uint32_t phase = 0, prev_phase = 0, mean_empty_phase = 1;
+    float* mean_out = p.mean + (int64_t)w.t * p.d + w.s * SE + ctid;
     for (int q = 0; q < Q; ++q) {
-        const int slot = q % kNBuf;
-        const uint32_t phase = (uint32_t)((q / kNBuf) & 1);
         const bool halo_tile = halo && q == 0;
         // the 128 threads leave together: a thread that saw a failed wait tells the others here
         bool bad = *sm.abort_flag != 0;
@@ -328,19 +329,25 @@ __device__ __forceinline__ void column_role(const CUtensorMap* tmap, const Fused
                 for (int gidx = 0; gidx < kColGroups; ++gidx) sum += sm.cs[gidx * SE + ctid];
                 const float m = sum / (float)p.f;
                 // the buffer was last used two tiles ago: wait until every row warp has read it
-                if (n >= 2 && !mbar_wait(sm.mean_empty + (n & 1), (uint32_t)(((n >> 1) + 1) & 1))) *sm.abort_flag = 1;
-                sm.mean_s[(n & 1) * SE + ctid] = m;
-                p.mean[(int64_t)w.t * p.d + w.s * SE + ctid] = m;
+                if (n >= 2 && !mbar_wait(sm.mean_empty + mb, mean_empty_phase)) *sm.abort_flag = 1;
+                sm.mean_s[mb * SE + ctid] = m;
+                *mean_out = m;
             }
             asm volatile("bar.sync 1, %0;" ::"n"(kColThreads) : "memory");
-            if (ctid == 0) mbar_arrive(sm.mean_full + (n & 1));
-            w.step(p);
+            if (ctid == 0) mbar_arrive(sm.mean_full + mb);
+            if (mb) mean_empty_phase ^= 1;              // units n and n+1 share a phase of their buffers
+            mb ^= 1;
+            if (w.step(p)) mean_out = p.mean + w.s * SE + ctid;
+            else mean_out += p.d;
         }
         // refill the buffer of the tile in front of this one as soon as every warp has let go of it
         if (ctid == 0 && q >= 1 && q - 1 + kNBuf < Q) {
-            if (mbar_wait(sm.empty + ((q - 1) % kNBuf), (uint32_t)(((q - 1) / kNBuf) & 1))) issue(q - 1 + kNBuf);
+            if (mbar_wait(sm.empty + prev_slot, prev_phase)) issue(prev_slot);
             else *sm.abort_flag = 1;                            // everyone leaves at the next check
         }
+        prev_slot = slot;
+        prev_phase = phase;
+        if (++slot == kNBuf) { slot = 0; phase ^= 1; }
     }
 }
 
@@ -467,31 +474,36 @@ __device__ __forceinline__ void row_role(const FusedParams& p, Smem<DT>& sm, int
         q = 1;
         has_prev = true;
     }
+    static_assert(kNBuf >= 2, "the halo tile and the first unit need their own buffers");
     Walk w;
     w.start(p, u0);
-    for (int n = 0; n < n_units; ++n, ++q) {
-        const int slot = q % kNBuf;
+    // ring position of the tile, mean buffer of the unit and the unit's record block, kept incrementally
+    int slot = q, mb = 0;
+    uint32_t phase = 0, mean_phase = 0;
+    const unsigned char* tile = sm.tiles + (size_t)slot * p.tile_stride;
+    const int64_t rec_step = (int64_t)p.nsl * p.f;
+    float4* rec_block = p.part + ((int64_t)w.t * p.nsl + w.s) * p.f;
+    for (int n = 0; n < n_units; ++n) {
         // a warp leaves as a whole: the lanes agree on what they saw
-        const bool fine = *sm.abort_flag == 0 && mbar_wait(sm.full + slot, (uint32_t)((q / kNBuf) & 1)) &&
-                          mbar_wait(sm.mean_full + (n & 1), (uint32_t)((n >> 1) & 1));
+        const bool fine = *sm.abort_flag == 0 && mbar_wait(sm.full + slot, phase) &&
+                          mbar_wait(sm.mean_full + mb, mean_phase);
         if (!__all_sync(0xffffffffu, fine)) {
             *sm.abort_flag = 1;
             return;
         }
         f32x2 m[2][H];
-        const float* ms = sm.mean_s + (n & 1) * SE;
+        const float* ms = sm.mean_s + mb * SE;
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
             for (int i = 0; i < H; ++i)
                 m[h][i] = *reinterpret_cast<const f32x2*>(ms + (st.j + 8 * h) * P + 2 * i);
         __syncwarp();
-        if (lane == 0) mbar_arrive(sm.mean_empty + (n & 1));
+        if (lane == 0) mbar_arrive(sm.mean_empty + mb);
 
         float x[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) x[i] = 0.f;
-        const unsigned char* tile = sm.tiles + (size_t)slot * p.tile_stride;
         if (has_prev && !w.is_first) st.template tile_pass<true>(tile, m, x);
         else st.template tile_pass<false>(tile, m, x);
         __syncwarp();
@@ -500,11 +512,19 @@ __device__ __forceinline__ void row_role(const FusedParams& p, Smem<DT>& sm, int
         // per-row sums of the slice: reduce over the row's 8 lanes, one record per row
         group8_reduce_scatter(x, st.j);
         const int row = st.slot_row(st.j >> 1);
-        if (row < p.f) {
-            float2* rec = reinterpret_cast<float2*>(p.part + ((int64_t)w.t * p.nsl + w.s) * p.f + row);
-            rec[st.j & 1] = make_float2(x[0], x[1]);    // even lane: ||a||^2, ||a-m||^2; odd: ||a-b||^2, ||b||^2
+        if (row < p.f)      // even lane: ||a||^2, ||a-m||^2; odd lane: ||a-b||^2, ||b||^2
+            reinterpret_cast<float2*>(rec_block + row)[st.j & 1] = make_float2(x[0], x[1]);
+        if (w.step(p)) {                                // a new slice starts without a previous frame
+            has_prev = false;
+            rec_block = p.part + (int64_t)w.s * p.f;
+        } else {
+            has_prev = true;
+            rec_block += rec_step;
         }
-        has_prev = !w.step(p);                          // a new slice starts without a previous frame
+        if (mb) mean_phase ^= 1;
+        mb ^= 1;
+        tile += p.tile_stride;
+        if (++slot == kNBuf) { slot = 0; phase ^= 1; tile = sm.tiles; }
     }
 }
 
