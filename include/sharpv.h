@@ -100,7 +100,8 @@ sharpv_status sharpv_score_frames(
 
 /* ------------------------------------------------------------------------------------------
  * Stage one (b): per-frame top-k and gather of the kept tokens.  Section 3.1 (first paragraph)
- * and 3.1.3 (last paragraph): "top-K selection of token importance scores" per frame.
+ * and 3.1.3 (last paragraph): in every frame the highest-scoring tokens are retained, as many as
+ * the frame's adaptive ratio allows.
  *
  * In frame t the k[t] tokens that come first under (importance descending, token index
  * ascending) are kept; -0 and +0 compare equal; NaN scores are not supported.  k[t] is
@@ -205,15 +206,14 @@ sharpv_status sharpv_kv_calibrate_prune_noalloc(
 
 /* ------------------------------------------------------------------------------------------
  * Stage two (b): K/V compaction.  Section 3.2.3: the discarded tokens' K/V is dropped so that
- * decoding only reads what was retained (Section 1, "retain visual tokens for subsequent
- * generation steps").
+ * decoding only reads the visual tokens that were retained (Section 1).
  *
  * For every layer in [layer_begin, layer_end), for K and V, for every KV head:
  *     dst[j, :] = src[kept_pos[j], :]      for j < n_kept = kept_seq_offsets[num_seqs]
  * as a bit copy of head_dim elements.  Strides are in elements; the head_dim axis is
  * contiguous; every stride * sizeof(element) and head_dim * sizeof(element) must be a
- * multiple of 16 bytes.  The benchmarked layout is [L][2][H][T][D_h]; a token-major cache is
- * expressed through the strides.  kv_dst == kv_src with identical strides compacts in place (every
+ * multiple of 16 bytes; a row (head_dim elements) may be at most 16 KB.  The benchmarked layout is
+ * [L][2][H][T][D_h]; a token-major cache is expressed through the strides.  kv_dst == kv_src with identical strides compacts in place (every
  * plane is walked front to back; serving stacks that cannot afford a second cache use this);
  * otherwise dst must not overlap src.  Rows of dst at and beyond
  * n_kept are left untouched.  `capacity` is an upper bound on n_kept that the host knows
