@@ -18,8 +18,8 @@
  *
  * Readings of the paper where it is silent (each is a convention; the tests pin
  * the arithmetic around them, not the choice itself):
- *   - first frame of a video: T_1 := S_1, the "virtual preceding frame made of the
- *     frame mean" of Section 3.1.3, so Eq. 6 is Eq. 5 applied to that T_1;
+ *   - first frame of a video: T_1 := S_1 (Section 3.1.3 treats the first frame as if a frame made
+ *     of its own mean stood in front of it), so Eq. 6 is Eq. 5 applied to that T_1;
  *   - the threshold of Eq. 5/6 is a retention ratio: k_t = round(threshold_t * f)
  *     followed by a per-frame top-k_t on I (Section 3.1.3, last paragraph);
  *   - ties in the top-k go to the lower token index; kept indices are reported
