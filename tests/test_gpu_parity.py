@@ -397,6 +397,113 @@ def test_nearly_parallel_rows_and_frame_sizes(dtype, d, grid):
     check_budgets(to_host(g["k"]), o, f)
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_score_random_shapes(seed):
+    """Random frame sizes, feature sizes, video counts (videos without frames included) and both
+    storage types: exercises every way a CTA's range of tiles can start, cross a slice and end."""
+    rng = np.random.default_rng(1000 + seed)
+    bf16 = bool(rng.integers(2))
+    f = int(rng.choice([1, 2, 3, 5, 17, 64, 100, 144, 169, 196, 201, 255, 256]))
+    slices = int(rng.choice([1, 2, 3, 7, 28]))
+    d = slices * (128 if bf16 else 64)
+    counts = [int(c) for c in rng.choice([0, 1, 1, 2, 3, 5, 9, 20], size=int(rng.integers(1, 7)))]
+    if sum(counts) == 0:
+        counts[0] = 4
+    vfo = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    F = int(vfo[-1])
+    x = rng.standard_normal((F * f, d)).astype(np.float32)
+    for t in range(1, F):                          # correlate consecutive frames, some exact duplicates
+        r = rng.random()
+        if r < 0.2:
+            x[t * f:(t + 1) * f] = x[(t - 1) * f:t * f]
+        elif r < 0.8:
+            x[t * f:(t + 1) * f] = 0.9 * x[(t - 1) * f:t * f] + 0.436 * x[t * f:(t + 1) * f]
+    xs = W.f32_to_bf16_bits(x) if bf16 else x
+    w = float(rng.choice([0.0, 0.5, 1.0, 2.0]))
+    o = orc.score_frames(xs, vfo, f, w=w, nthreads=NT)
+    g = sv.sharpv_score_frames(to_dev(xs), torch.from_numpy(vfo).cuda(), F, f, w=w, want_spatial=True,
+                               want_temporal=True)
+    torch.cuda.synchronize()
+    for key in ("spatial", "temporal", "importance", "ratio"):
+        e = rel_err(to_host(g[key]), o[key])
+        assert e <= TIGHT_TOL, f"{key}: rel err {e} (f={f}, d={d}, frames={counts}, bf16={bf16})"
+    check_budgets(to_host(g["k"]), o, f)
+    # selection on the GPU's own scores and budgets against the oracle's selection of the same inputs
+    sel = sv.sharpv_select_tokens(g["importance"], g["k"], F, f, gather=False)
+    torch.cuda.synchronize()
+    idx_o, off_o = orc.select_tokens(to_host(g["importance"]), to_host(g["k"]), f)
+    np.testing.assert_array_equal(to_host(sel["kept_offsets"]), off_o)
+    np.testing.assert_array_equal(to_host(sel["kept_index"])[:off_o[-1]], idx_o)
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_stage_two_random_layouts(seed):
+    """Random sequence layouts (system tokens before the visual block, sequences without visual tokens,
+    empty sequences), feature sizes, K/V shapes and cache layouts, out of place and in place."""
+    rng = np.random.default_rng(2000 + seed)
+    bf16 = bool(rng.integers(2))
+    d = int(rng.choice([8, 64, 200, 896])) * (1 if bf16 else 1)
+    B = int(rng.integers(1, 6))
+    n_sys = rng.integers(0, 4, B)
+    n_vis = rng.choice([0, 1, 7, 40, 300], size=B)
+    n_txt = rng.integers(0, 6, B)
+    if rng.random() < 0.3:
+        n_sys[-1] = n_vis[-1] = n_txt[-1] = 0              # a sequence without any token
+    lens = n_sys + n_vis + n_txt
+    if lens.sum() == 0:
+        n_vis[0], lens[0] = 5, 5
+    so = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    vo = np.concatenate([[0], np.cumsum(n_vis)])[:-1].astype(np.int32)
+    T, NV = int(so[-1]), int(n_vis.sum())
+    vis = rng.standard_normal((max(NV, 1), d)).astype(np.float32)
+    hid = rng.standard_normal((T, d)).astype(np.float32)
+    for b in range(B):
+        s0 = so[b] + n_sys[b]
+        drift = rng.uniform(0, 2, n_vis[b]).astype(np.float32)[:, None]
+        hid[s0:s0 + n_vis[b]] = vis[vo[b]:vo[b] + n_vis[b]] + drift * hid[s0:s0 + n_vis[b]]
+    if bf16:
+        vis, hid = W.f32_to_bf16_bits(vis), W.f32_to_bf16_bits(hid)
+    M = float(rng.choice([0.2, 0.6, 0.788, 0.95]))
+    vb, vc = n_sys.astype(np.int32), n_vis.astype(np.int32)
+    o = orc.kv_calibrate_prune(hid, vis, so, vb, vc, vo, M)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).cuda()
+    g = sv.sharpv_kv_calibrate_prune(to_dev(hid), to_dev(vis), i32(so), i32(vb), i32(vc), i32(vo), T, M=M,
+                                     want_mean_cos=True)
+    torch.cuda.synchronize()
+    if NV:
+        assert rel_err(to_host(g["cos"])[:NV], o["cos"][:NV]) <= TIGHT_TOL
+    kso = to_host(g["kept_seq_offsets"])
+    n = int(kso[-1])
+    kept = to_host(g["kept_pos"])[:n]
+    sym = np.setxor1d(kept, o["kept_pos"])
+    assert sym.size <= 1
+    if sym.size == 0:
+        np.testing.assert_array_equal(kso, o["kept_seq_offsets"])
+
+    L, H, Dh = int(rng.integers(1, 4)), int(rng.integers(1, 4)), int(rng.choice([8, 16, 64, 128]))
+    store = np.uint16 if bf16 else np.float32
+    token_major = bool(rng.integers(2))
+    shape = (L, 2, T, H, Dh) if token_major else (L, 2, H, T, Dh)
+    raw = (rng.integers(0, 65536, shape).astype(np.uint16) if bf16
+           else rng.standard_normal(shape).astype(np.float32))
+    kv_h = raw.transpose(0, 1, 3, 2, 4) if token_major else raw            # [L,2,H,T,Dh] view
+    kv_d = to_dev(raw)
+    kv_v = kv_d.permute(0, 1, 3, 2, 4) if token_major else kv_d
+    dst = torch.zeros((L, 2, H, max(n, 1) + 3, Dh), dtype=kv_d.dtype, device="cuda")
+    sv.sharpv_kv_compact(kv_v, dst, g["kept_pos"], g["kept_seq_offsets"], capacity=T)
+    torch.cuda.synchronize()
+    out = to_host(dst)
+    np.testing.assert_array_equal(out[:, :, :, :n], kv_h[:, :, :, kept])
+    assert not out[:, :, :, n:].any()
+    sv.sharpv_kv_compact(kv_v, kv_v, g["kept_pos"], g["kept_seq_offsets"], capacity=T)        # in place
+    torch.cuda.synchronize()
+    expect = np.ascontiguousarray(kv_h).copy()
+    orc.kv_compact_inplace(expect, kept)
+    got = to_host(kv_d)
+    np.testing.assert_array_equal(got.transpose(0, 1, 3, 2, 4) if token_major else got, expect)
+    assert store == got.dtype
+
+
 def test_run_to_run_bit_reproducible():
     wl, dw = _case("small_ragged")
     F, f = wl.total_frames, wl.f
