@@ -191,11 +191,14 @@ gather_rows_kernel(const char* __restrict__ src, int64_t src_row_bytes, int nvec
     const int lane = threadIdx.x & 31;
     const int64_t w = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int64_t j = w >> 1;
+    if (j >= capacity) return;
+    // the count and the index are fetched together (slot j exists even when it holds no index yet)
+    const int32_t row_index = __ldg(index + j);
     const int64_t n = min((int64_t)__ldg(count_ptr), capacity);
     if (j >= n) return;
     const int half = (nvec + 1) >> 1;
     const int v0 = (int)(w & 1) * half, v1 = min(nvec, v0 + half);
-    const char* s = src + (int64_t)__ldg(index + j) * src_row_bytes;
+    const char* s = src + (int64_t)row_index * src_row_bytes;
     char* o = dst + j * dst_row_bytes;
     for (int v = v0 + lane; v < v1; v += 256) {
         uint4 r[8];
