@@ -51,7 +51,9 @@ typedef enum {
     SHARPV_ERR_TIMEOUT = 6        /* (status_word only) a bounded device-side wait gave up */
 } sharpv_status;
 
-typedef enum { SHARPV_F32 = 0, SHARPV_BF16 = 1 } sharpv_dtype;
+/* SHARPV_U8 (any one-byte element, e.g. an fp8 K/V cache) is accepted by sharpv_kv_compact only: rows are
+ * copied bit for bit, never interpreted.  Scores and cosines need SHARPV_F32 or SHARPV_BF16. */
+typedef enum { SHARPV_F32 = 0, SHARPV_BF16 = 1, SHARPV_U8 = 2 } sharpv_dtype;
 
 /* How threshold_t * f (Eq. 5, 6) becomes an integer budget.  The paper is silent;
  * FLOOR never keeps more than the computed ratio and is the default of the binding. */

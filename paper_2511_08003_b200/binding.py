@@ -28,7 +28,7 @@ class Status(enum.IntEnum):
     ERR_TIMEOUT = 6
 
 
-F32, BF16 = 0, 1
+F32, BF16, U8 = 0, 1, 2
 ROUND_FLOOR, ROUND_NEAREST, ROUND_CEIL = 0, 1, 2
 DISSIM, ONE_MINUS_COS = 0, 1
 
@@ -150,10 +150,12 @@ def _workspace(ws: Optional[torch.Tensor], nbytes: int, device) -> torch.Tensor:
 
 
 def kv_layout(kv: torch.Tensor) -> KVLayout:
-    """Layout struct of a 5-D view [L, 2, H, T, D_h] (any strides, contiguous last axis)."""
+    """Layout struct of a 5-D view [L, 2, H, T, D_h] (any strides, contiguous last axis).  One-byte
+    caches (uint8 / int8 / fp8 tensors) are described as U8: compaction only copies bits."""
     if kv.dim() != 5 or kv.shape[1] != 2 or kv.stride(4) != 1:
         raise ValueError("K/V cache must be a [L, 2, H, T, D_h] view with a contiguous last axis")
-    return KVLayout(kv.shape[0], kv.shape[2], kv.shape[4], _dtype_code(kv),
+    code = U8 if kv.element_size() == 1 else _dtype_code(kv)
+    return KVLayout(kv.shape[0], kv.shape[2], kv.shape[4], code,
                     kv.stride(0), kv.stride(1), kv.stride(2), kv.stride(3))
 
 

@@ -16,8 +16,9 @@ constexpr float kNormEps = 1e-12f;      // v^ = v / max(||v||, kNormEps)
 // host-side argument checks
 // ---------------------------------------------------------------------------------------
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-inline int elem_bytes(sharpv_dtype dt) { return dt == SHARPV_F32 ? 4 : 2; }
+inline int elem_bytes(sharpv_dtype dt) { return dt == SHARPV_F32 ? 4 : (dt == SHARPV_BF16 ? 2 : 1); }
 inline bool dtype_ok(sharpv_dtype dt) { return dt == SHARPV_F32 || dt == SHARPV_BF16; }
+inline bool copy_dtype_ok(sharpv_dtype dt) { return dtype_ok(dt) || dt == SHARPV_U8; }    // bit copies only
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 inline sharpv_status launch_status() {

@@ -126,7 +126,7 @@ kv_compact_inplace_kernel(char* __restrict__ kv, PlaneGeom g, const int32_t* __r
 }
 
 bool layout_ok(const sharpv_kv_layout* L) {
-    return L && L->num_layers >= 1 && L->num_kv_heads >= 1 && L->head_dim >= 1 && dtype_ok(L->dtype) &&
+    return L && L->num_layers >= 1 && L->num_kv_heads >= 1 && L->head_dim >= 1 && copy_dtype_ok(L->dtype) &&
            L->stride_layer >= 0 && L->stride_kv >= 0 && L->stride_head >= 0 && L->stride_token >= L->head_dim;
 }
 
@@ -146,7 +146,7 @@ extern "C" sharpv_status sharpv_kv_compact(
     int32_t layer_begin, int32_t layer_end, const int32_t* kept_pos, const int32_t* kept_seq_offsets,
     int32_t num_seqs, int64_t capacity, int32_t* status_word, void* cuda_stream) {
     if (!layout_ok(src_layout) || !layout_ok(dst_layout)) {
-        if (src_layout && dst_layout && (!dtype_ok(src_layout->dtype) || !dtype_ok(dst_layout->dtype)))
+        if (src_layout && dst_layout && (!copy_dtype_ok(src_layout->dtype) || !copy_dtype_ok(dst_layout->dtype)))
             return SHARPV_ERR_UNSUPPORTED;
         return SHARPV_ERR_INVALID_ARG;
     }

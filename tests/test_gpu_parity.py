@@ -283,6 +283,31 @@ def test_layer_wise_reading_of_eq7():
     assert counts[0] > counts[-1] >= wl.n_text
 
 
+def test_kv_compact_one_byte_cache():
+    """An fp8-sized cache (one byte per element, 128-byte rows): compaction is a bit copy and needs no
+    knowledge of the element format."""
+    rng = np.random.default_rng(91)
+    L, H, T, Dh = 3, 4, 1500, 128
+    kv = rng.integers(0, 256, (L, 2, H, T, Dh), dtype=np.uint8)
+    kept = np.sort(rng.choice(T, size=600, replace=False)).astype(np.int32)
+    kept_d = torch.from_numpy(kept).cuda()
+    kso = torch.tensor([0, kept.size], dtype=torch.int32, device="cuda")
+    src = torch.from_numpy(kv).cuda()
+    dst = torch.zeros_like(src)
+    sv.sharpv_kv_compact(src, dst, kept_d, kso, capacity=T)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(dst.cpu().numpy(), orc.kv_compact(kv, kept))
+    sv.sharpv_kv_compact(src, src, kept_d, kso, capacity=T)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(src.cpu().numpy(), orc.kv_compact_inplace(kv.copy(), kept))
+    if hasattr(torch, "float8_e4m3fn"):
+        f8 = torch.from_numpy(kv).cuda().view(torch.float8_e4m3fn)
+        out = torch.zeros_like(f8)
+        sv.sharpv_kv_compact(f8, out, kept_d, kso, capacity=T)
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(out.view(torch.uint8).cpu().numpy()[:, :, :, :kept.size], kv[:, :, :, kept])
+
+
 def test_capacity_overflow_is_reported_not_written():
     wl, dw = _case("tiny")
     F, f, T = wl.total_frames, wl.f, wl.total_seq_tokens
