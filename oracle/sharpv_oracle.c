@@ -335,3 +335,49 @@ int sharpv_oracle_kv_compact_inplace(void *kv, int num_kv_heads, int64_t row_byt
     free(copy);
     return 0;
 }
+
+/*
+ * K/V compaction with positional re-encoding (Section 4.1.4: the positional embedding is encoded
+ * again when Memory SharpV prunes inside the LLM).  Reading, the paper giving no detail: the cached
+ * keys carry a rotary embedding of their old position (half-split pairing: dimension i pairs with
+ * i + rotary_dim/2, angle position * base^(-2i/rotary_dim)); a kept token moves from position
+ * p_old = kept_pos[j] - seq_offsets[b] to p_new = j - kept_seq_offsets[b] inside its sequence b, so
+ * its key is rotated by (p_new - p_old): x1' = x1 cos - x2 sin, x2' = x2 cos + x1 sin.  Values and
+ * the dimensions beyond rotary_dim are copied unchanged.  Output in double (the caller compares
+ * with the storage rounding in mind).  out: [L', 2, H, n_kept, D_h] dense, L' = layer_end - layer_begin.
+ */
+int sharpv_oracle_kv_compact_rope(const void *src, int dtype, int num_kv_heads, int head_dim,
+                                  int64_t stride_layer, int64_t stride_kv, int64_t stride_head,
+                                  int64_t stride_token, int layer_begin, int layer_end,
+                                  const int32_t *kept_pos, const int32_t *kept_seq_offsets,
+                                  const int32_t *seq_offsets, int num_seqs, int rotary_dim, double base,
+                                  double *out)
+{
+    if (rotary_dim < 0 || rotary_dim > head_dim || rotary_dim % 2) return -1;
+    int64_t n_kept = kept_seq_offsets[num_seqs];
+    int half = rotary_dim / 2;
+    int64_t o = 0;
+    for (int l = layer_begin; l < layer_end; ++l)
+        for (int kv = 0; kv < 2; ++kv)
+            for (int h = 0; h < num_kv_heads; ++h)
+                for (int b = 0; b < num_seqs; ++b)
+                    for (int64_t j = kept_seq_offsets[b]; j < kept_seq_offsets[b + 1]; ++j) {
+                        int64_t row = l * stride_layer + kv * stride_kv + h * stride_head +
+                                      (int64_t)kept_pos[j] * stride_token;       /* in elements */
+                        double delta = (double)(j - kept_seq_offsets[b]) -
+                                       (double)(kept_pos[j] - seq_offsets[b]);
+                        for (int i = 0; i < head_dim; ++i) {
+                            double x = load_elem(src, dtype, row + i);
+                            if (kv == 0 && i < rotary_dim) {
+                                int f = i < half ? i : i - half;
+                                double ang = delta * pow(base, -2.0 * f / rotary_dim);
+                                double partner = load_elem(src, dtype, row + (i < half ? i + half : i - half));
+                                x = i < half ? x * cos(ang) - partner * sin(ang)
+                                             : x * cos(ang) + partner * sin(ang);
+                            }
+                            out[o++] = x;
+                        }
+                    }
+    (void)n_kept;
+    return 0;
+}

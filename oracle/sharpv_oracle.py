@@ -201,3 +201,27 @@ def kv_compact_inplace(kv: np.ndarray, kept_pos, layer_begin: int = 0, layer_end
     if rc != 0:
         raise RuntimeError("sharpv_oracle_kv_compact_inplace failed")
     return kv
+
+
+def kv_compact_rope(kv_src: np.ndarray, kept_pos, kept_seq_offsets, seq_offsets, rotary_dim: int, base: float,
+                    layer_begin: int = 0, layer_end: Optional[int] = None) -> np.ndarray:
+    """Compaction with rotary re-encoding of the keys.  Returns float64 [L', 2, H, n_kept, D_h]."""
+    assert kv_src.ndim == 5 and kv_src.strides[4] == kv_src.itemsize
+    kp = np.ascontiguousarray(kept_pos, dtype=np.int32)
+    kso = np.ascontiguousarray(kept_seq_offsets, dtype=np.int32)
+    so = np.ascontiguousarray(seq_offsets, dtype=np.int32)
+    L, _, H, T, Dh = kv_src.shape
+    if layer_end is None:
+        layer_end = L
+    n = int(kso[-1])
+    out = np.empty((layer_end - layer_begin, 2, H, n, Dh), np.float64)
+    it = kv_src.itemsize
+    st = [x // it for x in kv_src.strides]
+    fn = lib().sharpv_oracle_kv_compact_rope
+    fn.restype = C.c_int
+    rc = fn(_ptr(kv_src), C.c_int(_dtype_code(kv_src)), C.c_int(H), C.c_int(Dh), C.c_int64(st[0]), C.c_int64(st[1]),
+            C.c_int64(st[2]), C.c_int64(st[3]), C.c_int(layer_begin), C.c_int(layer_end), _ptr(kp), _ptr(kso),
+            _ptr(so), C.c_int(so.size - 1), C.c_int(rotary_dim), C.c_double(base), _ptr(out))
+    if rc != 0:
+        raise RuntimeError("sharpv_oracle_kv_compact_rope failed")
+    return out

@@ -410,6 +410,48 @@ def test_kv_compact_inplace_equals_out_of_place_prefix():
     np.testing.assert_array_equal(tm[1][:, :kept.size], ref[1][:, :, kept].transpose(0, 2, 1, 3))
 
 
+def test_rope_reencoding_pins():
+    """Rotary re-encoding of compacted keys: (1) tokens that do not move are untouched and values never
+    change; (2) keys built as R(p_old) k come out as R(p_new) k; (3) pair norms are preserved;
+    (4) dimensions beyond rotary_dim are copied."""
+    rng = np.random.default_rng(36)
+    L, H, Dh, R, base = 2, 2, 16, 12, 10000.0
+    so = np.array([0, 9, 20], np.int32)                      # two sequences of 9 and 11 tokens
+    T = 20
+    kept = np.array([0, 1, 2, 5, 8, 9, 10, 14, 19], np.int32)
+    kso = np.array([0, 5, 9], np.int32)
+    half = R // 2
+    inv = base ** (-2.0 * np.arange(half) / R)
+
+    def rot(x, pos):                                         # textbook rotary embedding, half-split pairs
+        ang = np.asarray(pos, np.float64)[..., None] * inv
+        x1, x2 = x[..., :half], x[..., half:R]
+        return np.concatenate([x1 * np.cos(ang) - x2 * np.sin(ang), x2 * np.cos(ang) + x1 * np.sin(ang), x[..., R:]],
+                              axis=-1)
+
+    raw = rng.standard_normal((L, 2, H, T, Dh))
+    pos_old = np.concatenate([np.arange(9), np.arange(11)])
+    cache = raw.copy()
+    cache[:, 0] = rot(raw[:, 0], pos_old)                    # keys carry their old positions
+    cache32 = cache.astype(np.float32)
+    out = orc.kv_compact_rope(cache32, kept, kso, so, R, base)
+    pos_new = np.concatenate([np.arange(5), np.arange(4)])
+    expect_k = rot(raw[:, 0][:, :, kept], pos_new)
+    np.testing.assert_allclose(out[:, 0], expect_k, atol=2e-6)            # fp32 storage of the cache
+    np.testing.assert_array_equal(out[:, 1], cache32[:, 1][:, :, kept].astype(np.float64))   # values: bit copy
+    # tokens 0, 1, 2 of sequence 0 and token 9 (first of sequence 1) keep their positions
+    for j in (0, 1, 2, 5):
+        np.testing.assert_array_equal(out[:, 0, :, j], cache32[:, 0, :, kept[j]].astype(np.float64))
+    np.testing.assert_array_equal(out[:, 0, :, :, R:], cache32[:, 0][:, :, kept][..., R:].astype(np.float64))
+    kin = cache32[:, 0][:, :, kept].astype(np.float64)
+    n_in = np.hypot(kin[..., :half], kin[..., half:R])
+    n_out = np.hypot(out[:, 0][..., :half], out[:, 0][..., half:R])
+    np.testing.assert_allclose(n_out, n_in, rtol=1e-12)
+    # rotary_dim = 0 is plain compaction
+    np.testing.assert_array_equal(orc.kv_compact_rope(cache32, kept, kso, so, 0, base),
+                                  cache32[:, :, :, kept].astype(np.float64))
+
+
 def test_multithreaded_oracle_is_identical():
     wl = W.fill_hidden(W.fill_tokens(W.custom("mt", 34, W.BF16, 4, 64, 5, [W.make_video_spec(6, 0.9, cuts=[3])])))
     a = orc.score_frames(wl.tokens, wl.video_frame_offsets, wl.f, nthreads=1)
