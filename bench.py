@@ -51,6 +51,8 @@ def parse_args():
                          "(L2 flushed before each) and print its mean duration")
     ap.add_argument("--inplace", action="store_true",
                     help="compact the K/V cache in place (kv_dst == kv_src) instead of into a second cache")
+    ap.add_argument("--rope", action="store_true",
+                    help="compact with rotary re-encoding of the keys (rotary_dim = head_dim, base 1e6)")
     ap.add_argument("--layers", type=int, default=None,
                     help="override the number of K/V layers (profiling aid: smaller device footprint)")
     ap.add_argument("--frames", type=int, default=None,
@@ -303,7 +305,14 @@ def run_sharpv(args):
                                      tabs["vis_begin"], tabs["vis_count"], tabs["vis_offsets"], T, M=args.M,
                                      capacity=T, out=o_cal, workspace=ws_cal, status_word=status)
 
+    ws_rope = (torch.empty(sv.sharpv_kv_compact_rope_workspace_bytes(T, wl.head_dim), dtype=torch.uint8, device=dev)
+               if args.rope else None)
+
     def stage_compact(i=0):
+        if args.rope:
+            sv.sharpv_kv_compact_rope(kv, kv_dst, o_cal["kept_pos"], o_cal["kept_seq_offsets"], tabs["seq_offsets"],
+                                      T, wl.head_dim, 1.0e6, workspace=ws_rope, status_word=status)
+            return
         sv.sharpv_kv_compact(kv, kv if args.inplace else kv_dst, o_cal["kept_pos"], o_cal["kept_seq_offsets"],
                              capacity=T, status_word=status)
 
@@ -465,7 +474,7 @@ def run_sharpv(args):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "frames": F, "tokens_per_frame": f, "d": d, "storage": wl.dtype,
                    "visual_tokens": NV, "seq_tokens": T, "kv": list(wl.kv_shape()), "M": args.M, "w": args.w,
-                   "kept_stage_one": n_keep, "kept_stage_two": t_keep, "kv_in_place": bool(args.inplace),
+                   "kept_stage_one": n_keep, "kept_stage_two": t_keep, "kv_in_place": bool(args.inplace), "kv_rope": bool(args.rope),
                    "launch": "one CUDA graph replay per step, steps back to back",
                    "l2": "inputs larger than L2: a step streams several times the 126 MB L2 (K/V alone is "
                          "larger), and the per-kernel timings rotate through input copies totalling more than "

@@ -237,6 +237,32 @@ sharpv_status sharpv_kv_compact(
     const int32_t* kept_pos, const int32_t* kept_seq_offsets, int32_t num_seqs,
     int64_t capacity, int32_t* status_word, void* cuda_stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Stage two (b) with positional re-encoding.  Section 4.1.4 states that the positional embedding is
+ * encoded again when Memory SharpV prunes inside the LLM; it gives no detail, so this entry point fixes
+ * a reading: the cached keys carry a rotary embedding of their old position (half-split pairing:
+ * dimension i pairs with i + rotary_dim/2, angle position * rope_base^(-2i/rotary_dim)).  A kept token
+ * moves from p_old = kept_pos[j] - seq_offsets[b] to p_new = j - kept_seq_offsets[b] inside its
+ * sequence b, so while its key row is copied it is rotated by (p_new - p_old):
+ *     x1' = x1 cos - x2 sin,  x2' = x2 cos + x1 sin.
+ * Angles are evaluated in fp64, the rotation in fp32, the result is rounded to the storage type (round
+ * to nearest even).  Values and the dimensions at and beyond rotary_dim are bit copies; rotary_dim = 0
+ * is the plain compaction.  Same arguments as sharpv_kv_compact plus seq_offsets [dev] int32[num_seqs+1]
+ * (the packed sequence table of sharpv_kv_calibrate_prune), rotary_dim (even, <= head_dim,
+ * (rotary_dim / 2) * sizeof(element) a multiple of 16 bytes), rope_base > 0 and a workspace of
+ * sharpv_kv_compact_rope_workspace_bytes() bytes [dev] for the cos / sin table.  Out of place only;
+ * SHARPV_F32 and SHARPV_BF16 caches; rows of at most 8 KB.
+ */
+size_t sharpv_kv_compact_rope_workspace_bytes(int64_t capacity, int32_t rotary_dim);
+
+sharpv_status sharpv_kv_compact_rope(
+    const void* kv_src, const sharpv_kv_layout* src_layout /* [host] */,
+    void* kv_dst, const sharpv_kv_layout* dst_layout /* [host] */,
+    int32_t layer_begin, int32_t layer_end,
+    const int32_t* kept_pos, const int32_t* kept_seq_offsets, const int32_t* seq_offsets, int32_t num_seqs,
+    int64_t capacity, int32_t rotary_dim, double rope_base,
+    void* workspace, size_t workspace_bytes, int32_t* status_word, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

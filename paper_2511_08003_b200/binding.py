@@ -56,6 +56,7 @@ EXPORTS = (
     "sharpv_kv_calibrate_prune_workspace_bytes", "sharpv_kv_calibrate_prune",
     "sharpv_kv_calibrate_prune_noalloc",
     "sharpv_kv_compact",
+    "sharpv_kv_compact_rope_workspace_bytes", "sharpv_kv_compact_rope",
 )
 
 NOALLOC_MAX_SEQ_TOKENS = 262144
@@ -102,6 +103,11 @@ def lib():
     L.sharpv_kv_compact.restype = C.c_int
     L.sharpv_kv_compact.argtypes = [vp, C.POINTER(KVLayout), vp, C.POINTER(KVLayout), i32, i32, vp, vp, i32, i64,
                                     vp, vp]
+    L.sharpv_kv_compact_rope_workspace_bytes.restype = sz
+    L.sharpv_kv_compact_rope_workspace_bytes.argtypes = [i64, i32]
+    L.sharpv_kv_compact_rope.restype = C.c_int
+    L.sharpv_kv_compact_rope.argtypes = [vp, C.POINTER(KVLayout), vp, C.POINTER(KVLayout), i32, i32, vp, vp, vp, i32,
+                                         i64, i32, C.c_double, vp, sz, vp, vp]
     _lib = L
     return L
 
@@ -329,4 +335,27 @@ def sharpv_kv_compact(kv_src: torch.Tensor, kv_dst: torch.Tensor, kept_pos: torc
         _dev(kept_pos, "kept_pos", torch.int32), _dev(kept_seq_offsets, "kept_seq_offsets", torch.int32),
         kept_seq_offsets.numel() - 1, capacity, _dev(status_word, "status_word", torch.int32), _stream(stream))
     _check("sharpv_kv_compact", rc)
+    return kv_dst
+
+
+def sharpv_kv_compact_rope_workspace_bytes(capacity: int, rotary_dim: int) -> int:
+    return int(lib().sharpv_kv_compact_rope_workspace_bytes(capacity, rotary_dim))
+
+
+def sharpv_kv_compact_rope(kv_src: torch.Tensor, kv_dst: torch.Tensor, kept_pos: torch.Tensor,
+                           kept_seq_offsets: torch.Tensor, seq_offsets: torch.Tensor, capacity: int,
+                           rotary_dim: int, rope_base: float, layer_begin: int = 0,
+                           layer_end: Optional[int] = None, workspace=None, status_word=None,
+                           stream=None) -> torch.Tensor:
+    """Compaction with rotary re-encoding of the keys (values are bit copies).  Returns kv_dst."""
+    sl, dl = kv_layout(kv_src), kv_layout(kv_dst)
+    if layer_end is None:
+        layer_end = kv_src.shape[0]
+    ws = _workspace(workspace, sharpv_kv_compact_rope_workspace_bytes(capacity, rotary_dim), kv_src.device)
+    rc = lib().sharpv_kv_compact_rope(
+        _dev(kv_src, "kv_src"), C.byref(sl), _dev(kv_dst, "kv_dst"), C.byref(dl), layer_begin, layer_end,
+        _dev(kept_pos, "kept_pos", torch.int32), _dev(kept_seq_offsets, "kept_seq_offsets", torch.int32),
+        _dev(seq_offsets, "seq_offsets", torch.int32), kept_seq_offsets.numel() - 1, capacity, int(rotary_dim),
+        float(rope_base), ws.data_ptr(), ws.numel(), _dev(status_word, "status_word", torch.int32), _stream(stream))
+    _check("sharpv_kv_compact_rope", rc)
     return kv_dst

@@ -308,6 +308,50 @@ def test_kv_compact_one_byte_cache():
         np.testing.assert_array_equal(out.view(torch.uint8).cpu().numpy()[:, :, :, :kept.size], kv[:, :, :, kept])
 
 
+@pytest.mark.parametrize("dtype,Dh,R", [(W.BF16, 128, 128), (W.BF16, 128, 64), (W.F32, 64, 32), (W.F32, 64, 64),
+                                         (W.BF16, 64, 0)])
+def test_kv_compact_with_rotary_reencoding(dtype, Dh, R):
+    """Keys are rotated by the distance they move, values are bit copies.  The result is compared with the
+    fp64 oracle: fp32 caches to fp32 rounding, bf16 caches to half a bf16 ulp plus the fp32 error."""
+    rng = np.random.default_rng(92)
+    L, H = 2, 3
+    so = np.array([0, 700, 700, 1500, 1530], np.int32)           # four sequences, one of them empty
+    T = int(so[-1])
+    kept = np.sort(rng.choice(T, size=600, replace=False)).astype(np.int32)
+    kept[:40] = np.arange(40)                                    # a run that does not move at all
+    kept = np.unique(kept)
+    kso = np.searchsorted(kept, so).astype(np.int32)
+    raw = rng.standard_normal((L, 2, H, T, Dh)).astype(np.float32)
+    kv = W.f32_to_bf16_bits(raw) if dtype == W.BF16 else raw
+    base = 1.0e6
+    o = orc.kv_compact_rope(kv, kept, kso, so, R, base)
+    src = to_dev(kv)
+    cap = kept.size + 7
+    dst = torch.zeros((L, 2, H, cap, Dh), dtype=src.dtype, device="cuda")
+    i32 = lambda a: torch.from_numpy(a).cuda()
+    sv.sharpv_kv_compact_rope(src, dst, i32(kept), i32(kso), i32(so), cap, R, base)
+    torch.cuda.synchronize()
+    out = to_host(dst)
+    n = kept.size
+    assert not out[:, :, :, n:].any()                              # nothing written beyond the kept prefix
+    np.testing.assert_array_equal(out[:, 1, :, :n], kv[:, 1][:, :, kept])          # values: bit copy
+    np.testing.assert_array_equal(out[:, 0, :, :n, R:], kv[:, 0][:, :, kept][..., R:])   # beyond the rotary part
+    got = (W.bf16_bits_to_f32(out) if dtype == W.BF16 else out).astype(np.float64)[:, 0, :, :n, :R]
+    want = o[:, 0, :, :, :R]
+    if R:
+        half = R // 2
+        pair = np.hypot(want[..., :half], want[..., half:])
+        pair = np.concatenate([pair, pair], axis=-1)
+        # bf16 keeps 8 significant bits: half a unit in the last place is at most 2^-8 of the value
+        half_ulp = 2.0 ** -8 if dtype == W.BF16 else 0.0
+        assert np.all(np.abs(got - want) <= half_ulp * np.abs(want) * 1.001 + 4e-6 * pair + 1e-30)
+        moved = np.nonzero(kept - so[np.searchsorted(so, kept, side="right") - 1] !=
+                           np.arange(n) - kso[np.searchsorted(so, kept, side="right") - 1])[0]
+        assert moved.size > 100                                    # most tokens do move
+        still = np.setdiff1d(np.arange(n), moved)
+        np.testing.assert_array_equal(out[:, 0][:, :, still], kv[:, 0][:, :, kept[still]])   # unmoved keys: bit copy
+
+
 def test_capacity_overflow_is_reported_not_written():
     wl, dw = _case("tiny")
     F, f, T = wl.total_frames, wl.f, wl.total_seq_tokens

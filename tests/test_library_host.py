@@ -153,6 +153,34 @@ def test_kv_compact_rejects_bad_arguments(L):
     assert L.sharpv_kv_compact(P, None, 2 * P, None, 0, 1, P, P, 1, 10, None, None) == S.ERR_INVALID_ARG
 
 
+def test_kv_compact_rope_rejects_bad_arguments(L):
+    def layout(**kw):
+        base = dict(num_layers=2, num_kv_heads=4, head_dim=128, dtype=1, stride_layer=2 * 4 * 1000 * 128,
+                    stride_kv=4 * 1000 * 128, stride_head=1000 * 128, stride_token=128)
+        base.update(kw)
+        return sv.KVLayout(**base)
+
+    def call(src=P, sl=None, dst=2 * P, dl=None, lb=0, le=2, kp=P, kso=P, so=P, B=1, cap=1000, rd=128, rb=1e6,
+             ws=P, wsb=1 << 20):
+        sl = layout() if sl is None else sl
+        dl = layout() if dl is None else dl
+        return L.sharpv_kv_compact_rope(src, C.byref(sl), dst, C.byref(dl), lb, le, kp, kso, so, B, cap, rd, rb, ws,
+                                        wsb, None, None)
+
+    S = sv.Status
+    assert L.sharpv_kv_compact_rope_workspace_bytes(1000, 128) >= 1000 * 64 * 8
+    assert call(so=None) == S.ERR_INVALID_ARG
+    assert call(dst=P) == S.ERR_INVALID_ARG                       # out of place only
+    assert call(rd=130) == S.ERR_INVALID_ARG
+    assert call(rd=63) == S.ERR_INVALID_ARG                       # odd
+    assert call(rb=0.0) == S.ERR_INVALID_ARG
+    assert call(rd=8) == S.ERR_UNSUPPORTED                        # half a pair narrower than 16 bytes
+    assert call(sl=layout(dtype=2), dl=layout(dtype=2)) == S.ERR_UNSUPPORTED     # one-byte caches cannot be rotated
+    assert call(wsb=64) == S.ERR_WORKSPACE
+    assert call(ws=None) == S.ERR_INVALID_ARG
+    assert call(lb=1, le=1) == S.OK
+
+
 def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     monkeypatch.setattr(sv, "_lib", None)
     monkeypatch.setattr(sv._build, "LIB_PATH", str(tmp_path / "libsharpv.so"))
