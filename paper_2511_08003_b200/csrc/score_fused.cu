@@ -534,9 +534,11 @@ score_pass_kernel(const __grid_constant__ CUtensorMap tmap, const FusedParams p,
     extern __shared__ __align__(1024) unsigned char smem[];
     Smem<DT> sm(smem, p.tile_stride);
 
-    // let the finaliser's CTAs be scheduled as soon as SMs free up; they wait for this whole grid
-    cudaTriggerProgrammaticLaunchCompletion();
     cudaGridDependencySynchronize();        // the tokens come from earlier work on the stream
+    // Let the finaliser's CTAs be scheduled as soon as SMs free up; they wait for this whole grid.
+    // Only after the wait above: what the finaliser reads before its own wait (the frame table) is
+    // then known to be complete.
+    cudaTriggerProgrammaticLaunchCompletion();
     const int64_t U = (int64_t)p.nsl * p.F;
     const int64_t u0 = U * blockIdx.x / gridDim.x;
     const int64_t u1 = U * (blockIdx.x + 1) / gridDim.x;
