@@ -135,6 +135,41 @@ def test_select_alone_is_bit_exact_with_ties():
         np.testing.assert_array_equal(to_host(g2["kept_index"])[:off_o2[-1]], idx_o2)
 
 
+def test_random_selectors_of_the_ablation():
+    """The two random selectors of the ablation (Section 4.3.1: random choice under the per-frame
+    budgets of the method, and random choice video-wide under the total budget only) are the
+    per-frame top-k run on random scores; the random numbers are inputs, drawn on the host."""
+    wl, dw = _case("tiny")
+    F, f = wl.total_frames, wl.f
+    o = orc.score_frames(wl.tokens, wl.video_frame_offsets, f, w=1.0, nthreads=NT)
+    g = sv.sharpv_score_frames(dw.tokens, dw.video_frame_offsets, F, f, w=1.0)
+    torch.cuda.synchronize()
+    check_budgets(to_host(g["k"]), o, f)
+    rnd = np.random.default_rng(77).random(F * f).astype(np.float32)
+    d_rnd = torch.from_numpy(rnd).cuda()
+    # per-frame budgets of the method, random tokens inside each frame
+    k = to_host(g["k"])
+    s1 = sv.sharpv_select_tokens(d_rnd, g["k"], F, f, tokens=dw.tokens)
+    torch.cuda.synchronize()
+    idx_o, off_o = orc.select_tokens(rnd, k, f)
+    n = int(s1["num_kept"].item())
+    assert n == int(k.sum())
+    np.testing.assert_array_equal(to_host(s1["kept_offsets"]), off_o)
+    np.testing.assert_array_equal(to_host(s1["kept_index"])[:n], idx_o)
+    np.testing.assert_array_equal(to_host(s1["tokens"])[:n], wl.tokens[idx_o])
+    # one budget for the whole video: the video is one segment of F * f tokens
+    k_all = np.array([int(k.sum())], np.int32)
+    s2 = sv.sharpv_select_tokens(d_rnd, torch.from_numpy(k_all).cuda(), 1, F * f, tokens=dw.tokens)
+    torch.cuda.synchronize()
+    idx_o2, off_o2 = orc.select_tokens(rnd, k_all, F * f)
+    assert int(s2["num_kept"].item()) == n
+    np.testing.assert_array_equal(to_host(s2["kept_index"])[:n], idx_o2)
+    np.testing.assert_array_equal(to_host(s2["tokens"])[:n], wl.tokens[idx_o2])
+    # the same number of tokens, spread differently over the frames
+    per_frame = np.bincount(idx_o2 // f, minlength=F)
+    assert per_frame.sum() == n and not np.array_equal(per_frame, k)
+
+
 def test_select_threshold_variant():
     wl, dw = _case("tiny")
     F, f = wl.total_frames, wl.f
