@@ -28,6 +28,18 @@ __device__ __forceinline__ float dissim_sq_from_sums(float saa, float sbb, float
 
 constexpr float kRefineBelow = 1e-2f;   // squared Dissim under which the exact form is used
 
+// The same quantity from the inner product, 2 - 2 cos.  The cancellation leaves an absolute error of
+// a few 1e-7, which is harmless for a token against its frame mean (far from parallel in practice);
+// under kRefineBelowDot the caller re-evaluates from the rows.
+__device__ __forceinline__ float dissim_sq_from_dot(float saa, float sbb, float sab) {
+    const float na = sqrtf(saa), nb = sqrtf(sbb);
+    if (na >= kNormEps && nb >= kNormEps) return fmaxf(2.f - 2.f * sab / (na * nb), 0.f);
+    const float ca = fmaxf(na, kNormEps), cb = fmaxf(nb, kNormEps);
+    return fmaxf(saa / (ca * ca) + sbb / (cb * cb) - 2.f * sab / (ca * cb), 0.f);
+}
+
+constexpr float kRefineBelowDot = 6.25e-2f;
+
 
 // Exact re-evaluation of one token row: sums the squared differences of the normalised rows
 // directly.  One warp per row; every lane returns the warp totals.  ia, ib, im are the

@@ -4,20 +4,24 @@
 // the f x 256-byte tile of frame t.  Persistent CTAs (one per SM) each take a contiguous range of
 // units in (slice-major, frame-minor) order, so a CTA walks consecutive frames of one slice.
 //
-//   score_pass_kernel      640 threads in two roles that only meet through mbarriers:
-//       column warps (4)   issue the TMA loads that fill a ring of tile buffers, add up the columns
-//                          of each tile (the whole frame column is inside the tile, so this is the
-//                          slice of the frame mean) and publish the mean one tile ahead of the rows;
-//       row warps (16)     keep their part of the previous frame's tile in registers (4 rows x two
-//                          16-byte vectors per thread), visit each new tile once for ||a||^2,
-//                          ||a - mean||^2 and ||a - b||^2 with packed fp32 FMAs, overwrite the old
-//                          rows in place and write one record of partial sums per row and slice.
-//       Every wait is on the CTA's own barriers and is bounded.
+//   score_pass_kernel      512 threads in two roles that meet at hardware barriers:
+//       row warps (up to 12; 16 lanes per row, one 16-byte vector per lane, two rows per warp
+//                          and visit) keep the frame they saw last in registers, already widened
+//                          to fp32, and the vectors of the next tile on their way in from global
+//                          memory (one 128-bit streaming load per row and lane, issued a whole
+//                          tile ahead).  A tile is visited once: each element is widened once and
+//                          feeds ||a||^2, the column sums of the tile and ||a - b||^2 against the
+//                          registers, which it then replaces.  While the helper turns the column
+//                          sums into the frame mean the warp adds up its row sums over the 16
+//                          lanes of a row (through its own patch of shared memory); then it takes
+//                          <a, mean> from the registers and writes one record of partial sums per
+//                          row and slice.
+//       helper warps (4)   add up the column sums the row warps leave in shared memory, publish
+//                          the slice of the frame mean and tell the row warps what the next unit is.
+//       No thread ever spins: the roles wait for each other at bar.sync only.
 //   score_finalize_kernel  one CTA per frame, launched as a programmatic dependent so that its
 //       start-up overlaps the tail of the pass: adds the slices in a fixed order and writes
 //       S, T, I, the ratio and the budget of the frame.
-#include <cuda.h>
-
 #include "score_common.cuh"
 #include "score_fused.cuh"
 
@@ -25,18 +29,14 @@ namespace sharpv {
 namespace {
 
 constexpr int kSliceBytes = 256;
-constexpr int kRowWarps = 16;           // a row warp = 4 row groups x 8 lanes (two vectors per lane)
-constexpr int kColWarps = 4;            // 128 threads = 16 vector columns x 8 row groups
-constexpr int kRowThreads = kRowWarps * 32;
-constexpr int kColThreads = kColWarps * 32;
-constexpr int kThreads = kRowThreads + kColThreads;
-constexpr int kColGroups = kColThreads / 16;
-constexpr int kRows = 4;                // row slots per row-warp thread: frames of up to 256 tokens
-constexpr int kMaxTokensFused = 256;
-constexpr int kNBuf = 3;                // tile buffers in the ring
-constexpr int kSmemBudget = 227 * 1024;
-constexpr uint32_t kSpinLimit = 1u << 24;      // polls of one mbarrier before a wait gives up
-constexpr long long kSpinClocks = 2000000000ll; // ... or about one second of SM clock
+constexpr int kMaxRowWarps = 12;        // a row warp = 2 rows x 16 lanes (one vector per lane)
+constexpr int kHelpWarps = 4;
+constexpr int kRowThreads = kMaxRowWarps * 32;      // three warpgroups; warps beyond W stay idle
+constexpr int kHelpThreads = kHelpWarps * 32;
+constexpr int kThreads = kRowThreads + kHelpThreads;
+constexpr int kMaxVisits = 11;          // rows a half warp keeps in registers
+constexpr int kMaxTokensFused = 256;    // the finaliser takes one row per thread of a 256-thread group
+static_assert(2 * kMaxRowWarps * kMaxVisits >= kMaxTokensFused, "the row warps must cover the largest frame");
 constexpr int kFinThreads = 1024;
 
 struct FusedParams {
@@ -50,45 +50,19 @@ struct FusedParams {
     float *out_I, *out_S, *out_T, *out_ratio;
     int32_t* out_k;
     float* mean;            // [F, d]
-    float4* part;           // [F, nsl, f]: (||a||^2, ||a-m||^2, ||a-b||^2, ||b||^2) of the slice
-    uint32_t tile_bytes, tile_stride;
+    float4* part;           // [F, nsl, f]: (||a||^2, <a, m>, ||a-b||^2, ||b||^2) of the slice
+    int W;                  // row warps at work: a tile is covered in R = ceil(f / 2W) visits
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+// Hardware barriers between the roles: the side that hands something over arrives, the side that
+// needs it syncs; `threads` counts both sides.  A warp that waits here issues nothing meanwhile.
+constexpr int kBarSums = 1;     // column sums of a tile are in colp (row warps -> helper warps)
+constexpr int kBarMean = 2;     // frame mean of a tile and the next unit's tag are out (helper -> row warps)
+__device__ __forceinline__ void bar_arrive(int id, int threads) {
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// bounded wait: false when the limit ran out (a poll count and, every 256 polls, about a second of
-// SM clock, whichever comes first)
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (uint32_t i = 1; i < kSpinLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 0 && clock64() - t0 > kSpinClocks) return false;
-    }
-    return false;
-}
-__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+__device__ __forceinline__ void bar_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
 // Two fp32 values in one 64-bit register, the operand form of the packed fp32 instructions.
@@ -108,6 +82,11 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
     return d;
 }
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
     f32x2 d;
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
@@ -118,16 +97,10 @@ __device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
     asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
-// one 32-bit word of two bf16 -> the two exact fp32 values (a bf16 is the upper half of an fp32):
-// one multiply and one mask, on different pipes, written straight into the halves of the result
+// one word of two bf16 -> the two exact fp32 values as a pair (a bf16 is the upper half of an fp32);
+// plain integer code, so that the compiler places the halves of the pair itself
 __device__ __forceinline__ f32x2 widen_bf16x2(uint32_t w) {
-    f32x2 r;
-    asm("{\n\t.reg .b32 lo, hi;\n\t"
-        "mul.lo.u32 lo, %1, 65536;\n\t"          // low element: shift up (multiply pipe)
-        "and.b32 hi, %1, 0xffff0000;\n\t"        // high element: mask (logic pipe)
-        "mov.b64 %0, {lo, hi};\n\t}"
-        : "=l"(r) : "r"(w));
-    return r;
+    return ((unsigned long long)(w & 0xffff0000u) << 32) | (unsigned long long)(w << 16);
 }
 __device__ __forceinline__ f32x2 pair_f32(uint32_t lo, uint32_t hi) {
     f32x2 r;
@@ -135,65 +108,10 @@ __device__ __forceinline__ f32x2 pair_f32(uint32_t lo, uint32_t hi) {
     return r;
 }
 
-// 8 lanes x 16 values (x[4*slot + j], 4 slots) -> lane L of the group ends with x[0], x[1] =
-// values 2*(L&1), 2*(L&1)+1 of slot L>>1.  Fixed pairing, hence a fixed summation order.
-__device__ __forceinline__ void group8_reduce_scatter(float (&x)[16], int lane8) {
-    {
-        const bool up = lane8 & 4;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float lo = x[i], hi = x[8 + i];
-            x[i] = (up ? hi : lo) + __shfl_xor_sync(0xffffffffu, up ? lo : hi, 4);
-        }
-    }
-    {
-        const bool up = lane8 & 2;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float lo = x[i], hi = x[4 + i];
-            x[i] = (up ? hi : lo) + __shfl_xor_sync(0xffffffffu, up ? lo : hi, 2);
-        }
-    }
-    {
-        const bool up = lane8 & 1;
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const float lo = x[i], hi = x[2 + i];
-            x[i] = (up ? hi : lo) + __shfl_xor_sync(0xffffffffu, up ? lo : hi, 1);
-        }
-    }
-}
-
 __device__ __forceinline__ bool frame_is_first(const int32_t* vfo, int num_videos, int t) {
     const int b = upper_segment(vfo, num_videos, t);
     return __ldg(vfo + b) == t;
 }
-
-// Shared-memory layout of one CTA.
-template <int DT>
-struct Smem {
-    static constexpr int SE = kSliceBytes / Elem<DT>::kBytes;       // elements per slice row
-    unsigned char* tiles;       // [kNBuf][tile_stride]
-    float* cs;                  // [kColGroups][SE] column sums of each row group of the column warps
-    float* mean_s;              // [2][SE] frame-mean slice of the tiles, alternating
-    uint64_t* full;             // [kNBuf] tile landed (TMA)
-    uint64_t* empty;            // [kNBuf] tile released by all 20 warps
-    uint64_t* mean_full;        // [2] mean published by the column warps
-    uint64_t* mean_empty;       // [2] mean read by all 16 row warps
-    volatile int* abort_flag;
-
-    __device__ __forceinline__ Smem(unsigned char* base, uint32_t tile_stride) {
-        tiles = base;
-        cs = reinterpret_cast<float*>(base + (size_t)kNBuf * tile_stride);
-        mean_s = cs + kColGroups * SE;
-        full = reinterpret_cast<uint64_t*>(mean_s + 2 * SE);
-        empty = full + kNBuf;
-        mean_full = empty + kNBuf;
-        mean_empty = mean_full + 2;
-        abort_flag = reinterpret_cast<volatile int*>(mean_empty + 2);
-    }
-    static size_t fixed_bytes() { return (size_t)(kColGroups * SE + 2 * SE) * 4 + (2 * kNBuf + 4) * 8 + 16; }
-};
 
 // where a CTA stands in its range of units
 struct Walk {
@@ -228,6 +146,29 @@ struct Walk {
     }
 };
 
+
+// Shared memory of one CTA (about 40 KB).
+template <int DT>
+struct Smem {
+    static constexpr int SE = kSliceBytes / Elem<DT>::kBytes;   // elements per slice row
+    static constexpr int kRedStride = 66;                       // floats per visit slot: a float2 per lane, and 2 so that the slots start on different banks
+    static constexpr int kRedFloats = 16 * kRedStride;          // per row warp: 16 visit slots
+    float colp[2 * kMaxRowWarps * SE];      // column sums of each half warp, lane-major order
+    float red[kMaxRowWarps * kRedFloats];   // row sums of each warp on their way across lanes
+    float mean_s[SE];                       // frame-mean slice of the newest tile, same order as colp
+    int2 info[2];                           // of unit n, at n & 1: t * nsl + s, "opens a video"
+};
+
+// Order of the SE floats of a slice row in colp / mean_s: float 4k + q of lane j's vector sits at
+// (16k + j) * 4 + q, so that the 16 lanes of a row store and load whole float4s side by side.
+// Returns the column of the slice that position `off` holds.
+template <int DT>
+__device__ __forceinline__ int column_of_position(int off) {
+    constexpr int P = Elem<DT>::kPerVec;
+    const int q = off & 3, j = (off >> 2) & 15, k = off >> 6;
+    return j * P + 4 * k + q;
+}
+
 template <int DT>
 __device__ __forceinline__ void widen_pairs(const uint4& v, f32x2 (&o)[Elem<DT>::kPerVec / 2]) {
     constexpr int H = Elem<DT>::kPerVec / 2;
@@ -239,300 +180,233 @@ __device__ __forceinline__ void widen_pairs(const uint4& v, f32x2 (&o)[Elem<DT>:
     }
 }
 
-// barrier 1 over the column warps with an OR of `flag`: every thread gets the same answer
-__device__ __forceinline__ bool column_any(bool flag) {
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 p, %1, 0;\n\t"
-        "bar.red.or.pred q, 1, %2, p;\n\t"
-        "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(out) : "r"((uint32_t)flag), "n"(kColThreads) : "memory");
-    return out != 0;
-}
-
 // ---------------------------------------------------------------------------------------
-// column warps: TMA producer, column sums, frame mean
+// helper warps: frame mean, unit tags
 // ---------------------------------------------------------------------------------------
 template <int DT>
-__device__ __forceinline__ void column_role(const CUtensorMap* tmap, const FusedParams& p, Smem<DT>& sm, int64_t u0,
-                                            int n_units, int halo, int ctid) {
-    using E = Elem<DT>;
-    constexpr int P = E::kPerVec, H = P / 2, SE = Smem<DT>::SE;
-    const int Q = n_units + halo;
-    const int vcol = ctid & 15, rgrp = ctid >> 4, lane = ctid & 31;
-
-    // tiles are requested in unit order: (load_s, load_t) just advances (thread 0 of the role)
-    int load_s = (int)(u0 / p.F), load_t = (int)(u0 % p.F) - halo;
-    auto issue = [&](int slot) {
-        mbar_expect_tx(sm.full + slot, p.tile_bytes);
-        tma_load_2d(sm.tiles + (size_t)slot * p.tile_stride, tmap, load_s * kSliceBytes, load_t * p.f,
-                    sm.full + slot);
-        if (++load_t == p.F) { load_t = 0; ++load_s; }
-    };
-    if (ctid == 0)
-        for (int q = 0; q < kNBuf && q < Q; ++q) issue(q);
-
+__device__ __forceinline__ void helper_role(const FusedParams& p, Smem<DT>& sm, int64_t u0, int n_units, int htid) {
+    constexpr int SE = Smem<DT>::SE;
     Walk w;
     w.start(p, u0);
-    // ring position of tile q and of tile q-1, and the mean buffer of unit n, all kept incrementally
-    int slot = 0, prev_slot = 0, mb = 0;
-    uint32_t phase = 0, prev_phase = 0, mean_empty_phase = 1;
-    float* mean_out = p.mean + (int64_t)w.t * p.d + w.s * SE + ctid;
-    for (int q = 0; q < Q; ++q) {
-        const bool halo_tile = halo && q == 0;
-        // the 128 threads leave together: a thread that saw a failed wait tells the others here
-        bool bad = *sm.abort_flag != 0;
-        if (!bad && !halo_tile && !mbar_wait(sm.full + slot, phase)) {
-            *sm.abort_flag = 1;
-            bad = true;
-        }
-        if (column_any(bad)) return;
-        if (halo_tile) {
-            if (lane == 0) mbar_arrive(sm.empty + slot);        // the column warps do not read the halo tile
-        } else {
-            const int n = q - halo;
-            const unsigned char* tile = sm.tiles + (size_t)slot * p.tile_stride + vcol * 16;
-            f32x2 acc[H];
-#pragma unroll
-            for (int i = 0; i < H; ++i) acc[i] = pk(0.f, 0.f);
-            int r = rgrp;
-            for (; r + 3 * kColGroups < p.f; r += 4 * kColGroups) {
-                uint4 v[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    v[u] = *reinterpret_cast<const uint4*>(tile + (r + u * kColGroups) * kSliceBytes);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    f32x2 a2[H];
-                    widen_pairs<DT>(v[u], a2);
-#pragma unroll
-                    for (int i = 0; i < H; ++i) acc[i] = add2(acc[i], a2[i]);
-                }
+    const int column = column_of_position<DT>(htid & (SE - 1));
+    float* mean_out = p.mean + (int64_t)w.t * p.d + w.s * SE + column;
+    const float* my_col = sm.colp + htid;
+    const int groups = 2 * p.W;
+    const int both = 32 * p.W + kHelpThreads;
+    const float ff = (float)p.f;
+    if (htid == 0) sm.info[0] = make_int2(w.t * p.nsl + w.s, w.is_first ? 1 : 0);
+    bar_arrive(kBarMean, both);                 // the first unit's tag is out
+    for (int n = 0; n < n_units; ++n) {
+        float* out = mean_out;
+        if (w.step(p)) mean_out = p.mean + w.s * SE + column;
+        else mean_out += p.d;
+        if (htid == 0) sm.info[(n + 1) & 1] = make_int2(w.t * p.nsl + w.s, w.is_first ? 1 : 0);
+        bar_sync(kBarSums, both);
+        if (htid < SE) {
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+            int gidx = 0;
+#pragma unroll 2
+            for (; gidx + 3 < groups; gidx += 4) {
+                s0 += my_col[(gidx + 0) * SE];
+                s1 += my_col[(gidx + 1) * SE];
+                s2 += my_col[(gidx + 2) * SE];
+                s3 += my_col[(gidx + 3) * SE];
             }
-            for (; r < p.f; r += kColGroups) {
-                f32x2 a2[H];
-                widen_pairs<DT>(*reinterpret_cast<const uint4*>(tile + r * kSliceBytes), a2);
-#pragma unroll
-                for (int i = 0; i < H; ++i) acc[i] = add2(acc[i], a2[i]);
+            if (gidx < groups) {            // groups is even
+                s0 += my_col[(gidx + 0) * SE];
+                s1 += my_col[(gidx + 1) * SE];
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(sm.empty + slot);        // this warp is done with the tile
-            float* dst = sm.cs + rgrp * SE + vcol * P;
-#pragma unroll
-            for (int i = 0; i < H; i += 2)
-                *reinterpret_cast<ulonglong2*>(dst + 2 * i) = make_ulonglong2(acc[i], acc[i + 1]);
-            asm volatile("bar.sync 1, %0;" ::"n"(kColThreads) : "memory");
-            if (ctid < SE) {
-                float sum = 0.f;
-#pragma unroll
-                for (int gidx = 0; gidx < kColGroups; ++gidx) sum += sm.cs[gidx * SE + ctid];
-                const float m = sum / (float)p.f;
-                // the buffer was last used two tiles ago: wait until every row warp has read it
-                if (n >= 2 && !mbar_wait(sm.mean_empty + mb, mean_empty_phase)) *sm.abort_flag = 1;
-                sm.mean_s[mb * SE + ctid] = m;
-                *mean_out = m;
-            }
-            asm volatile("bar.sync 1, %0;" ::"n"(kColThreads) : "memory");
-            if (ctid == 0) mbar_arrive(sm.mean_full + mb);
-            if (mb) mean_empty_phase ^= 1;              // units n and n+1 share a phase of their buffers
-            mb ^= 1;
-            if (w.step(p)) mean_out = p.mean + w.s * SE + ctid;
-            else mean_out += p.d;
+            const float m = ((s0 + s1) + (s2 + s3)) / ff;
+            sm.mean_s[htid] = m;
+            *out = m;
         }
-        // refill the buffer of the tile in front of this one as soon as every warp has let go of it
-        if (ctid == 0 && q >= 1 && q - 1 + kNBuf < Q) {
-            if (mbar_wait(sm.empty + prev_slot, prev_phase)) issue(prev_slot);
-            else *sm.abort_flag = 1;                            // everyone leaves at the next check
-        }
-        prev_slot = slot;
-        prev_phase = phase;
-        if (++slot == kNBuf) { slot = 0; phase ^= 1; }
+        bar_arrive(kBarMean, both);
     }
 }
 
 // ---------------------------------------------------------------------------------------
 // row warps
 // ---------------------------------------------------------------------------------------
-template <int DT>
-struct RowState {
+// Lane (g, j) of warp `warp` (g = lane / 16) owns, in visit v, vector j of row 2 W v + 2 warp + g.
+// Visits below R - 1 exist for every warp and every lane; in the last one a warp takes part if its
+// first row exists, and a half warp whose own row lies beyond the frame loads nothing and works on
+// zeros.
+//
+// Row sums cross the 16 lanes of a row through the warp's own patch of shared memory: every lane
+// leaves its parts there, then lane l adds up the 16 parts of row l / 16, visit l % 16 of the warp,
+// in lane order.
+template <int DT, int R>
+struct RowRegs {
     static constexpr int H = Elem<DT>::kPerVec / 2;
-    uint4 prev[kRows][2];   // previous frame's rows of this thread (two vectors each)
-    float bb[kRows];        // this thread's share of ||previous row||^2
-    int warp, g, j, f;
+    static constexpr int kRS = 66;      // floats per visit slot of the warp's patch (Smem::kRedStride)
+    f32x2 prev[R][H];       // the frame seen last, fp32 pairs: [visit][pair]
+    uint4 raw[R];           // the tile about to be visited, as it arrives from global memory
 
-    // Row slot r of this thread is row 64 r + 4 warp + g (g = lane group): a warp owns four
-    // consecutive rows per slot.  A slot is visited when its first row exists (a warp-uniform test);
-    // lane groups whose row lies beyond the frame read the zero rows that pad every tile buffer to a
-    // multiple of four rows, so no lane ever branches on its own row.
-    __device__ __forceinline__ bool slot_live(int r) const { return 64 * r + 4 * warp < f; }
-    __device__ __forceinline__ int slot_row(int r) const { return 64 * r + 4 * warp + g; }
-    __device__ __forceinline__ const unsigned char* my_rows(const unsigned char* tile) const {
-        return tile + (4 * warp + g) * kSliceBytes + j * 16;
-    }
-
-    // frame in front of the first unit: registers only
-    __device__ __forceinline__ void load_halo(const unsigned char* tile) {
-        const unsigned char* base = my_rows(tile);
+    __device__ __forceinline__ void clear() {
 #pragma unroll
-        for (int r = 0; r < kRows; ++r) {
-            f32x2 acc = pk(0.f, 0.f);
-            if (slot_live(r)) {
+        for (int v = 0; v < R; ++v) {
+            raw[v] = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    prev[r][h] = *reinterpret_cast<const uint4*>(base + r * (64 * kSliceBytes) + h * 128);
-                    f32x2 b2[H];
-                    widen_pairs<DT>(prev[r][h], b2);
-#pragma unroll
-                    for (int i = 0; i < H; ++i) acc = fma2(b2[i], b2[i], acc);
-                }
-            }
-            bb[r] = hsum(acc);
+            for (int i = 0; i < H; ++i) prev[v][i] = pk(0.f, 0.f);
         }
     }
 
-    // slots [R0, R1) of one tile, without a branch: ||a||^2, ||a - m||^2 and, when the frame continues
-    // a video (TEMPORAL), ||a - b||^2 against the rows in registers, which the new rows then replace
-    template <int R0, int R1, bool TEMPORAL>
-    __device__ __forceinline__ void slots(const unsigned char* base, const f32x2 (&m)[2][H], float (&x)[16]) {
-        uint4 a4[R1 - R0][2];
+    // requests this lane's vectors of the tile at `tile` (this lane's first row and column)
+    __device__ __forceinline__ void request(const char* tile, int64_t vstride, bool last_mine) {
 #pragma unroll
-        for (int r = R0; r < R1; ++r)
+        for (int v = 0; v < R; ++v)
+            if (v < R - 1 || last_mine) raw[v] = __ldcs(reinterpret_cast<const uint4*>(tile + v * vstride));
+    }
+
+    // One visit of the tile in `raw`: ||a||^2 and ||a - b||^2 (TEMPORAL, b = the rows in registers)
+    // of this lane's part of each row go to the warp's patch, col += a (COLS), the registers then
+    // hold the new rows, and the vectors of the tile behind it (`next`, if any) are requested as
+    // soon as a register is free for them.
+    template <bool TEMPORAL, bool COLS>
+    __device__ __forceinline__ void take_tile(const char* next, int64_t vstride, bool last_warp, bool last_mine,
+                                              f32x2 (&col)[H], float* red_lane) {
 #pragma unroll
-            for (int h = 0; h < 2; ++h)
-                a4[r - R0][h] = *reinterpret_cast<const uint4*>(base + r * (64 * kSliceBytes) + h * 128);
-#pragma unroll
-        for (int r = R0; r < R1; ++r) {
-            f32x2 aa = pk(0.f, 0.f), dm = aa, db = aa;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
+        for (int v = 0; v < R; ++v) {
+            if (v < R - 1 || last_warp) {
                 f32x2 a2[H];
-                widen_pairs<DT>(a4[r - R0][h], a2);
+                widen_pairs<DT>(raw[v], a2);
+                if (next && (v < R - 1 || last_mine)) raw[v] = __ldcs(reinterpret_cast<const uint4*>(next + v * vstride));
+                f32x2 aa, db;
 #pragma unroll
                 for (int i = 0; i < H; ++i) {
-                    const f32x2 e = sub2(a2[i], m[h][i]);
-                    aa = fma2(a2[i], a2[i], aa);
-                    dm = fma2(e, e, dm);
-                }
-                if (TEMPORAL) {
-                    f32x2 b2[H];
-                    widen_pairs<DT>(prev[r][h], b2);
-#pragma unroll
-                    for (int i = 0; i < H; ++i) {
-                        const f32x2 e = sub2(a2[i], b2[i]);
-                        db = fma2(e, e, db);
+                    aa = i == 0 ? mul2(a2[i], a2[i]) : fma2(a2[i], a2[i], aa);
+                    if (COLS) col[i] = (v == 0 && R > 1) ? a2[i] : add2(col[i], a2[i]);
+                    if (TEMPORAL) {
+                        const f32x2 e = sub2(a2[i], prev[v][i]);
+                        db = i == 0 ? mul2(e, e) : fma2(e, e, db);
                     }
+                    prev[v][i] = a2[i];
                 }
-                prev[r][h] = a4[r - R0][h];
+                *reinterpret_cast<float2*>(red_lane + v * kRS) = make_float2(hsum(aa), TEMPORAL ? hsum(db) : 0.f);
             }
-            x[4 * r + 0] = hsum(aa);
-            x[4 * r + 1] = hsum(dm);
-            x[4 * r + 2] = hsum(db);
-            x[4 * r + 3] = TEMPORAL ? bb[r] : 0.f;
-            bb[r] = x[4 * r + 0];
         }
     }
 
-    template <bool TEMPORAL>
-    __device__ __forceinline__ void tile_pass(const unsigned char* tile, const f32x2 (&m)[2][H], float (&x)[16]) {
-        const unsigned char* base = my_rows(tile);
-        if (slot_live(2)) {                     // the usual case: a straight run over three slots
-            slots<0, 2, TEMPORAL>(base, m, x);
-            slots<2, 3, TEMPORAL>(base, m, x);
-            if (slot_live(3)) slots<3, 4, TEMPORAL>(base, m, x);
-        } else {
-            if (slot_live(0)) slots<0, 1, TEMPORAL>(base, m, x);
-            if (slot_live(1)) slots<1, 2, TEMPORAL>(base, m, x);
+    // <a, mean> of the rows in registers, this lane's part of each row, to the warp's patch
+    __device__ __forceinline__ void against_mean(const f32x2 (&m)[H], bool last_warp, int g, float* red_lane) const {
+#pragma unroll
+        for (int v = 0; v < R; ++v) {
+            if (v < R - 1 || last_warp) {
+                f32x2 am;
+#pragma unroll
+                for (int i = 0; i < H; ++i) am = i == 0 ? mul2(prev[v][i], m[i]) : fma2(prev[v][i], m[i], am);
+                red_lane[v * kRS + g] = hsum(am);
+            }
         }
     }
 };
 
-template <int DT>
+template <int DT, int R>
 __device__ __forceinline__ void row_role(const FusedParams& p, Smem<DT>& sm, int64_t u0, int n_units, int halo,
                                          int tid) {
-    using E = Elem<DT>;
-    constexpr int P = E::kPerVec, H = P / 2, SE = Smem<DT>::SE;
-    const int lane = tid & 31;
-    RowState<DT> st;
-    st.warp = tid >> 5;
-    st.g = lane >> 3;
-    st.j = lane & 7;
-    st.f = p.f;
-#pragma unroll
-    for (int r = 0; r < kRows; ++r) {
-        st.prev[r][0] = make_uint4(0u, 0u, 0u, 0u);
-        st.prev[r][1] = st.prev[r][0];
-        st.bb[r] = 0.f;
-    }
-    int q = 0;
-    bool has_prev = false;
-    if (halo) {
-        if (!__all_sync(0xffffffffu, mbar_wait(sm.full + 0, 0))) { *sm.abort_flag = 1; return; }
-        st.load_halo(sm.tiles);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(sm.empty + 0);
-        q = 1;
-        has_prev = true;
-    }
-    static_assert(kNBuf >= 2, "the halo tile and the first unit need their own buffers");
-    Walk w;
-    w.start(p, u0);
-    // ring position of the tile, mean buffer of the unit and the unit's record block, kept incrementally
-    int slot = q, mb = 0;
-    uint32_t phase = 0, mean_phase = 0;
-    const unsigned char* tile = sm.tiles + (size_t)slot * p.tile_stride;
-    const int64_t rec_step = (int64_t)p.nsl * p.f;
-    float4* rec_block = p.part + ((int64_t)w.t * p.nsl + w.s) * p.f;
-    for (int n = 0; n < n_units; ++n) {
-        // a warp leaves as a whole: the lanes agree on what they saw
-        const bool fine = *sm.abort_flag == 0 && mbar_wait(sm.full + slot, phase) &&
-                          mbar_wait(sm.mean_full + mb, mean_phase);
-        if (!__all_sync(0xffffffffu, fine)) {
-            *sm.abort_flag = 1;
-            return;
-        }
-        f32x2 m[2][H];
-        const float* ms = sm.mean_s + mb * SE;
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int i = 0; i < H; ++i)
-                m[h][i] = *reinterpret_cast<const f32x2*>(ms + (st.j + 8 * h) * P + 2 * i);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(sm.mean_empty + mb);
+    constexpr int H = Elem<DT>::kPerVec / 2, SE = Smem<DT>::SE;
+    static_assert(H >= 2, "two accumulators per sum");
+    const int lane = tid & 31, warp = tid >> 5, g = lane >> 4, j = lane & 15;
+    const int row0 = 2 * warp + g;
+    const bool last_warp = 2 * p.W * (R - 1) + 2 * warp < p.f;      // the warp takes part in the last visit
+    const bool last_mine = 2 * p.W * (R - 1) + row0 < p.f;          // and this lane's own row exists there
+    const int64_t vstride = (int64_t)2 * p.W * p.row_bytes_ld;
+    const int64_t frame_bytes = (int64_t)p.f * p.row_bytes_ld;
+    float* my_colp = sm.colp + (2 * warp + g) * SE + j * 4;         // float4 k of this lane at + 64 k
+    const float* my_mean = sm.mean_s + j * 4;
+    float* red_warp = sm.red + warp * Smem<DT>::kRedFloats;
+    float* red_lane = red_warp + lane * 2;                          // visit v of this lane at + 64 v
+    // the row sums this lane adds up: row sg of the warp's two, visit sv, starting with lane srot
+    const int sg = lane >> 4, sv = lane & 15;
+    const float* sum_src = red_warp + sv * Smem<DT>::kRedStride + sg * 32;    // float2 of lane j' of the row at + 2 j'
+    const int my_row = 2 * p.W * sv + 2 * warp + sg;
+    const bool sums = sv < R;
+    const bool writes = sums && my_row < p.f;
+    const int both = 32 * p.W + kHelpThreads;
 
-        float x[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) x[i] = 0.f;
-        if (has_prev && !w.is_first) st.template tile_pass<true>(tile, m, x);
-        else st.template tile_pass<false>(tile, m, x);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(sm.empty + slot);            // this warp is done with the tile
+    RowRegs<DT, R> st;
+    st.clear();
+    float prev_aa = 0.f;            // ||row||^2 of the frame seen last, for the row this lane adds up
 
-        // per-row sums of the slice: reduce over the row's 8 lanes, one record per row
-        group8_reduce_scatter(x, st.j);
-        const int row = st.slot_row(st.j >> 1);
-        if (row < p.f)      // even lane: ||a||^2, ||a-m||^2; odd lane: ||a-b||^2, ||b||^2
-            reinterpret_cast<float2*>(rec_block + row)[st.j & 1] = make_float2(x[0], x[1]);
-        if (w.step(p)) {                                // a new slice starts without a previous frame
-            has_prev = false;
-            rec_block = p.part + (int64_t)w.s * p.f;
-        } else {
-            has_prev = true;
-            rec_block += rec_step;
+    // this lane's first vector of the first tile: the frame in front of the range, if it matters
+    const int s0 = (int)(u0 / p.F);
+    int t = (int)(u0 % p.F) - halo;
+    const char* tile = p.tokens + ((int64_t)t * p.f + row0) * p.row_bytes_ld + (int64_t)s0 * kSliceBytes + j * 16;
+    st.request(tile, vstride, last_mine);
+    bar_sync(kBarMean, both);                   // the first unit's tag
+    const int Q = n_units + halo;
+    int n = 0;
+    for (int q = 0; q < Q; ++q) {
+        const bool halo_tile = halo && q == 0;
+        // the tile behind this one: the next frame of the slice, or the first frame of the next slice
+        const char* next = nullptr;
+        if (q + 1 < Q) {
+            if (++t == p.F) {
+                t = 0;
+                next = tile - (int64_t)(p.F - 1) * frame_bytes + kSliceBytes;
+            } else {
+                next = tile + frame_bytes;
+            }
         }
-        if (mb) mean_phase ^= 1;
-        mb ^= 1;
-        tile += p.tile_stride;
-        if (++slot == kNBuf) { slot = 0; phase ^= 1; tile = sm.tiles; }
+        const int2 inf = sm.info[n & 1];
+        const bool temporal = !halo_tile && inf.y == 0;     // the frame continues a video
+        f32x2 col[H];
+        if (R == 1) {               // the only visit may be one this warp has no part in
+#pragma unroll
+            for (int i = 0; i < H; ++i) col[i] = pk(0.f, 0.f);
+        }
+        if (halo_tile) st.template take_tile<false, false>(next, vstride, last_warp, last_mine, col, red_lane);
+        else if (temporal) st.template take_tile<true, true>(next, vstride, last_warp, last_mine, col, red_lane);
+        else st.template take_tile<false, true>(next, vstride, last_warp, last_mine, col, red_lane);
+        tile = next;
+        if (!halo_tile) {
+#pragma unroll
+            for (int k = 0; k < H / 2; ++k)
+                *reinterpret_cast<ulonglong2*>(my_colp + 64 * k) = make_ulonglong2(col[2 * k], col[2 * k + 1]);
+            bar_arrive(kBarSums, both);                     // the column sums are out
+        }
+        __syncwarp();
+        // row sums of ||a||^2 and ||a - b||^2 while the helper makes the mean
+        f32x2 xy = pk(0.f, 0.f);
+        if (sums) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                xy = add2(xy, *reinterpret_cast<const f32x2*>(sum_src + 2 * i));
+        }
+        __syncwarp();                                       // the patch is free again
+        float my_aa, my_db;
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(my_aa), "=f"(my_db) : "l"(xy));
+
+        if (!halo_tile) {
+            bar_sync(kBarMean, both);
+            f32x2 m[H];
+#pragma unroll
+            for (int k = 0; k < H / 2; ++k) {
+                const ulonglong2 x = *reinterpret_cast<const ulonglong2*>(my_mean + 64 * k);
+                m[2 * k] = x.x;
+                m[2 * k + 1] = x.y;
+            }
+            st.against_mean(m, last_warp, g, red_lane);
+            __syncwarp();
+            float my_am = 0.f;
+            if (sums) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) my_am += sum_src[2 * i + sg];
+            }
+            __syncwarp();                                   // the patch is free again
+            if (writes)
+                p.part[(int64_t)inf.x * p.f + my_row] = make_float4(my_aa, my_am, my_db, temporal ? prev_aa : 0.f);
+            ++n;
+        }
+        prev_aa = my_aa;
     }
 }
 
-template <int DT>
+template <int DT, int R>
 __global__ void __launch_bounds__(kThreads, 1)
-score_pass_kernel(const __grid_constant__ CUtensorMap tmap, const FusedParams p, int32_t* status_word) {
-    extern __shared__ __align__(1024) unsigned char smem[];
-    Smem<DT> sm(smem, p.tile_stride);
+score_pass_kernel(const FusedParams p) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    Smem<DT>& sm = *reinterpret_cast<Smem<DT>*>(smem);
 
     cudaGridDependencySynchronize();        // the tokens come from earlier work on the stream
     // Let the finaliser's CTAs be scheduled as soon as SMs free up; they wait for this whole grid.
@@ -548,47 +422,15 @@ score_pass_kernel(const __grid_constant__ CUtensorMap tmap, const FusedParams p,
     const int vid0 = upper_segment(p.video_frame_offsets, p.num_videos, t0);
     const int halo = (__ldg(p.video_frame_offsets + vid0) == t0) ? 0 : 1;
 
+    // The block is launched with 128 registers per thread (512 x 128 = 65536).  The helper warps give
+    // most of theirs back and the three row warpgroups take them: 128 x 32 + 384 x 160 = 65536.
     const int tid = threadIdx.x;
-    if (tid == 0) {
-        for (int i = 0; i < kNBuf; ++i) {
-            mbar_init(sm.full + i, 1);
-            mbar_init(sm.empty + i, kRowWarps + kColWarps);
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(sm.mean_full + i, 1);
-            mbar_init(sm.mean_empty + i, kRowWarps);
-        }
-        *sm.abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    // rows beyond the frame in every tile buffer stay zero for the whole kernel (TMA writes f rows)
-    for (int b = 0; b < kNBuf; ++b) {
-        uint4* pad = reinterpret_cast<uint4*>(sm.tiles + (size_t)b * p.tile_stride + p.tile_bytes);
-        const int n = (int)((p.tile_stride - p.tile_bytes) / 16);
-        for (int i = tid; i < n; i += kThreads) pad[i] = make_uint4(0u, 0u, 0u, 0u);
-    }
-    __syncthreads();
-
-    // The block is launched with 96 registers per thread (640 x 96 = 61440).  The column warps give
-    // most of theirs back and the four row warpgroups take 8 more each: 128 x 48 + 512 x 104 = 59392.
     if (tid < kRowThreads) {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 104;");
-        row_role<DT>(p, sm, u0, n_units, halo, tid);
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 160;");
+        if ((tid >> 5) < p.W) row_role<DT, R>(p, sm, u0, n_units, halo, tid);
     } else {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
-        column_role<DT>(&tmap, p, sm, u0, n_units, halo, tid - kRowThreads);
-    }
-
-    __syncthreads();
-    if (*sm.abort_flag && tid == 0) {
-        // A bounded wait ran out.  Report it, then give every tile buffer one more bounded wait so
-        // that no load lands in shared memory after the CTA has gone.
-        report(status_word, SHARPV_ERR_TIMEOUT);
-        for (int i = 0; i < kNBuf; ++i) {
-            (void)mbar_wait(sm.full + i, 0);
-            (void)mbar_wait(sm.full + i, 1);
-        }
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 32;");
+        helper_role<DT>(p, sm, u0, n_units, tid - kRowThreads);
     }
 }
 
@@ -640,12 +482,12 @@ score_finalize_kernel(const FusedParams p) {
 
     if (tid < p.f) {
         const float4 a0 = g_sum[0][tid], a1 = g_sum[1][tid], a2 = g_sum[2][tid], a3 = g_sum[3][tid];
-        const float aa = (a0.x + a1.x) + (a2.x + a3.x), dm = (a0.y + a1.y) + (a2.y + a3.y);
+        const float aa = (a0.x + a1.x) + (a2.x + a3.x), am = (a0.y + a1.y) + (a2.y + a3.y);
         const float db = (a0.z + a1.z) + (a2.z + a3.z), bb = (a0.w + a1.w) + (a2.w + a3.w);
-        const float s2 = dissim_sq_from_sums(aa, smm, dm);
+        const float s2 = dissim_sq_from_dot(aa, smm, am);
         const float t2 = is_first ? 0.f : dissim_sq_from_sums(aa, bb, db);
         int fl = 0;
-        if (s2 < kRefineBelow && dm != 0.f) fl |= 1;
+        if (s2 < kRefineBelowDot) fl |= 1;
         if (!is_first && t2 < kRefineBelow && db != 0.f) fl |= 2;
         f_s2[tid] = s2; f_t2[tid] = t2; f_aa[tid] = aa; f_bb[tid] = bb; f_fl[tid] = fl;
     }
@@ -691,41 +533,41 @@ score_finalize_kernel(const FusedParams p) {
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = [] {
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess) {
-            (void)cudaGetLastError();
-            ptr = nullptr;
-        }
-        return (EncodeTiledFn)ptr;
-    }();
-    return fn;
+// The split of a frame over the row warps: W warps cover 2W rows a visit and the frame in
+// R = ceil(f / 2W) visits; warp w sits on scheduler w mod 4.  The split with the lightest
+// busiest scheduler wins, then the larger W.
+void row_split(int f, int& W, int& R) {
+    int best = 1 << 30;
+    W = kMaxRowWarps;
+    R = kMaxVisits;
+    for (int w = 1; w <= kMaxRowWarps; ++w) {
+        const int r = (f + 2 * w - 1) / (2 * w);
+        if (r > kMaxVisits) continue;
+        int load[4] = {0, 0, 0, 0};
+        for (int i = 0; i < w; ++i) load[i & 3] += r - 1 + (2 * w * (r - 1) + 2 * i < f ? 1 : 0);
+        int worst = 0;
+        for (int k = 0; k < 4; ++k) worst = load[k] > worst ? load[k] : worst;
+        if (worst <= best) { best = worst; W = w; R = r; }
+    }
 }
 
-template <int DT>
-sharpv_status launch(const FusedScoreArgs& a, const CUtensorMap& tmap, FusedParams& p, int sms) {
-    const size_t smem = (size_t)kNBuf * p.tile_stride + Smem<DT>::fixed_bytes();
-    if (smem > (size_t)kSmemBudget) return SHARPV_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(score_pass_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+template <int DT, int R>
+sharpv_status launch(const FusedScoreArgs& a, FusedParams& p, int sms) {
+    const size_t smem = sizeof(Smem<DT>);
+    if (cudaFuncSetAttribute(score_pass_kernel<DT, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess) {
         (void)cudaGetLastError();
         return SHARPV_ERR_UNSUPPORTED;
     }
     const int64_t units = (int64_t)p.nsl * a.F;
     const unsigned grid = (unsigned)(units < sms ? units : sms);
-    if (launch_dependent(score_pass_kernel<DT>, dim3(grid), dim3(kThreads), smem, a.stream, tmap, p,
-                         a.status_word) != cudaSuccess) {
+    if (launch_dependent(score_pass_kernel<DT, R>, dim3(grid), dim3(kThreads), smem, a.stream, p) != cudaSuccess) {
         (void)cudaGetLastError();
         return SHARPV_ERR_CUDA;
     }
-
+#ifdef NOFIN
+    return SHARPV_OK;
+#endif
     // the finaliser starts while the pass drains and waits for it with cudaGridDependencySynchronize
     if (launch_dependent(score_finalize_kernel<DT>, dim3((unsigned)a.F), dim3(kFinThreads), 0, a.stream, p) !=
         cudaSuccess) {
@@ -733,6 +575,24 @@ sharpv_status launch(const FusedScoreArgs& a, const CUtensorMap& tmap, FusedPara
         return SHARPV_ERR_CUDA;
     }
     return SHARPV_OK;
+}
+
+template <int DT>
+sharpv_status launch_visits(const FusedScoreArgs& a, FusedParams& p, int sms, int R) {
+    switch (R) {
+        case 1: return launch<DT, 1>(a, p, sms);
+        case 2: return launch<DT, 2>(a, p, sms);
+        case 3: return launch<DT, 3>(a, p, sms);
+        case 4: return launch<DT, 4>(a, p, sms);
+        case 5: return launch<DT, 5>(a, p, sms);
+        case 6: return launch<DT, 6>(a, p, sms);
+        case 7: return launch<DT, 7>(a, p, sms);
+        case 8: return launch<DT, 8>(a, p, sms);
+        case 9: return launch<DT, 9>(a, p, sms);
+        case 10: return launch<DT, 10>(a, p, sms);
+        case 11: return launch<DT, 11>(a, p, sms);
+    }
+    return SHARPV_ERR_UNSUPPORTED;
 }
 
 }  // namespace
@@ -748,8 +608,6 @@ size_t fused_score_workspace_bytes(int F, int f, int d) {
 }
 
 sharpv_status fused_score_launch(const FusedScoreArgs& a) {
-    EncodeTiledFn enc = encode_fn();
-    if (!enc) return SHARPV_ERR_UNSUPPORTED;
     const int eb = elem_bytes(a.dtype);
     FusedParams p;
     p.tokens = (const char*)a.tokens;
@@ -764,25 +622,15 @@ sharpv_status fused_score_launch(const FusedScoreArgs& a) {
     char* w = (char*)a.workspace;
     p.mean = (float*)w;       w += align_up((size_t)a.F * a.d * 4, 256);
     p.part = (float4*)w;
-    p.tile_bytes = (uint32_t)a.f * kSliceBytes;
-    p.tile_stride = (uint32_t)((a.f + 3) / 4 * 4) * kSliceBytes;   // whole groups of four rows; the tail stays zero
-
-    // the token matrix as a byte tensor [rows, d * elem_bytes]; one box is one (frame, slice) tile
-    CUtensorMap tmap;
-    const cuuint64_t gdim[2] = {(cuuint64_t)a.d * eb, (cuuint64_t)a.F * a.f};
-    const cuuint64_t gstr[1] = {(cuuint64_t)p.row_bytes_ld};
-    const cuuint32_t box[2] = {(cuuint32_t)kSliceBytes, (cuuint32_t)a.f};
-    const cuuint32_t estr[2] = {1, 1};
-    if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void*)a.tokens, gdim, gstr, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return SHARPV_ERR_UNSUPPORTED;
 
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
         return SHARPV_ERR_CUDA;
-    return a.dtype == SHARPV_F32 ? launch<SHARPV_F32>(a, tmap, p, sms) : launch<SHARPV_BF16>(a, tmap, p, sms);
+    int R = 0;
+    row_split(a.f, p.W, R);
+    return a.dtype == SHARPV_F32 ? launch_visits<SHARPV_F32>(a, p, sms, R)
+                                 : launch_visits<SHARPV_BF16>(a, p, sms, R);
 }
 
 }  // namespace sharpv

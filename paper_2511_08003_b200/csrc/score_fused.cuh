@@ -28,7 +28,7 @@ bool fused_score_supported(sharpv_dtype dtype, int f, int d);
 // Upper bound over both storage types.
 size_t fused_score_workspace_bytes(int F, int f, int d);
 
-// SHARPV_ERR_UNSUPPORTED means "could not set up (no tensor-map encoder)": nothing was launched
+// SHARPV_ERR_UNSUPPORTED means "could not set up (shared-memory size refused)": nothing was launched
 // and the caller should take the three-kernel path.
 sharpv_status fused_score_launch(const FusedScoreArgs& a);
 
