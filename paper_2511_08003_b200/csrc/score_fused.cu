@@ -270,7 +270,8 @@ struct RowRegs {
             if (v < R - 1 || last_warp) {
                 f32x2 a2[H];
                 widen_pairs<DT>(raw[v], a2);
-                if (next && (v < R - 1 || last_mine)) raw[v] = __ldcs(reinterpret_cast<const uint4*>(next + v * vstride));
+                if (next && (v < R - 1 || last_mine)) raw[v] = __ldcs(reinterpret_cast<const uint4*>(next));
+                next += vstride;
                 f32x2 aa, db;
 #pragma unroll
                 for (int i = 0; i < H; ++i) {
