@@ -48,7 +48,7 @@ typedef enum {
     SHARPV_ERR_WORKSPACE = 3,     /* workspace smaller than the matching *_workspace_bytes() */
     SHARPV_ERR_CAPACITY = 4,      /* (status_word only) more survivors than `capacity` */
     SHARPV_ERR_CUDA = 5,          /* a CUDA runtime call or launch failed */
-    SHARPV_ERR_TIMEOUT = 6        /* (status_word only) a bounded device-side wait gave up */
+    SHARPV_ERR_TIMEOUT = 6        /* (status_word only) reserved: a bounded device-side wait gave up; no kernel waits that way at present */
 } sharpv_status;
 
 /* SHARPV_U8 (any one-byte element, e.g. an fp8 K/V cache) is accepted by sharpv_kv_compact only: rows are
