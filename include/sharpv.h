@@ -238,6 +238,38 @@ sharpv_status sharpv_kv_compact(
     int64_t capacity, int32_t* status_word, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Stage two read layer by layer.  Section 3.2.3 states Eq. 7 on the hidden state of a layer l and drops
+ * "the corresponding layer's" K/V; Table 1 lists the method as adaptive per layer and Section 1 calls the
+ * result a hierarchical cache pruning.  This entry point applies sharpv_kv_calibrate_prune and
+ * sharpv_kv_compact once per layer l in [layer_begin, layer_end): layer l is calibrated on its own
+ * hidden state and only its own K and V planes are compacted with its own kept list, so deeper layers
+ * may keep fewer tokens than shallow ones.
+ *
+ * hidden [dev]: the hidden states of the layers in the range, layer l at
+ *   hidden + (l - layer_begin) * stride_hidden_layer elements, each [total_seq_tokens, d] with row
+ *   stride ld_hidden; stride_hidden_layer * sizeof(element) must be a multiple of 16 bytes.
+ * Outputs are per layer, layer l at index i = l - layer_begin:
+ *   out_cos [dev] float[i * total_visual ...], out_mean_cos [dev] float[i * num_seqs ...] or NULL,
+ *   out_kept_pos [dev] int32[i * capacity ...], out_kept_seq_offsets [dev] int32[i * (num_seqs + 1) ...].
+ * kv_src / kv_dst and their layouts as in sharpv_kv_compact (kv_dst == kv_src compacts in place); rows of
+ * a layer's planes at and beyond that layer's kept count are left untouched.  All other arguments, the
+ * workspace (sharpv_kv_calibrate_prune_workspace_bytes, shared by the layers, which run one after the
+ * other on the stream) and the error behaviour are those of the two entry points it is made of.
+ */
+sharpv_status sharpv_kv_prune_layers(
+    const void* hidden, int64_t stride_hidden_layer, int64_t ld_hidden, const void* visual, int64_t ld_visual,
+    sharpv_dtype dtype, int32_t d,
+    int32_t num_seqs, const int32_t* seq_offsets, const int32_t* vis_begin,
+    const int32_t* vis_count, const int32_t* vis_offsets,
+    int64_t total_seq_tokens, int64_t total_visual, float M,
+    float* out_cos, float* out_mean_cos,
+    int32_t* out_kept_pos, int32_t* out_kept_seq_offsets, int64_t capacity,
+    const void* kv_src, const sharpv_kv_layout* src_layout /* [host] */,
+    void* kv_dst, const sharpv_kv_layout* dst_layout /* [host] */,
+    int32_t layer_begin, int32_t layer_end,
+    void* workspace, size_t workspace_bytes, int32_t* status_word, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
  * Stage two (b) with positional re-encoding.  Section 4.1.4 states that the positional embedding is
  * encoded again when Memory SharpV prunes inside the LLM; it gives no detail, so this entry point fixes
  * a reading: the cached keys carry a rotary embedding of their old position (half-split pairing:

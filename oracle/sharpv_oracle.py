@@ -203,6 +203,21 @@ def kv_compact_inplace(kv: np.ndarray, kept_pos, layer_begin: int = 0, layer_end
     return kv
 
 
+def kv_prune_layers(hidden_layers, visual: np.ndarray, seq_offsets, vis_begin, vis_count, vis_offsets, M: float,
+                    kv: np.ndarray, layer_begin: int = 0, nthreads: int = 0):
+    """Section 3.2.3 read layer by layer: Eq. 7 on the hidden state of each layer decides which of that
+    layer's K/V rows stay.  hidden_layers[i] is the hidden state of layer layer_begin + i.  Returns the
+    per-layer results of kv_calibrate_prune and a copy of kv whose planes of those layers are compacted
+    in place (rows at and beyond a layer's kept count keep their old contents)."""
+    out = np.array(kv, copy=True)
+    results = []
+    for i, h in enumerate(hidden_layers):
+        o = kv_calibrate_prune(h, visual, seq_offsets, vis_begin, vis_count, vis_offsets, M, nthreads=nthreads)
+        kv_compact_inplace(out, o["kept_pos"], layer_begin=layer_begin + i, layer_end=layer_begin + i + 1)
+        results.append(o)
+    return results, out
+
+
 def kv_compact_rope(kv_src: np.ndarray, kept_pos, kept_seq_offsets, seq_offsets, rotary_dim: int, base: float,
                     layer_begin: int = 0, layer_end: Optional[int] = None) -> np.ndarray:
     """Compaction with rotary re-encoding of the keys.  Returns float64 [L', 2, H, n_kept, D_h]."""

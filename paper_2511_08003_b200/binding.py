@@ -55,7 +55,7 @@ EXPORTS = (
     "sharpv_select_tokens_workspace_bytes", "sharpv_select_tokens", "sharpv_select_tokens_threshold",
     "sharpv_kv_calibrate_prune_workspace_bytes", "sharpv_kv_calibrate_prune",
     "sharpv_kv_calibrate_prune_noalloc",
-    "sharpv_kv_compact",
+    "sharpv_kv_prune_layers", "sharpv_kv_compact",
     "sharpv_kv_compact_rope_workspace_bytes", "sharpv_kv_compact_rope",
 )
 
@@ -100,6 +100,10 @@ def lib():
     L.sharpv_kv_calibrate_prune_noalloc.restype = C.c_int
     L.sharpv_kv_calibrate_prune_noalloc.argtypes = [vp, i64, vp, i64, C.c_int, i32, i32, vp, vp, vp, vp, i64, i64,
                                                     f32, vp, vp, vp, vp, i64, vp, vp]
+    L.sharpv_kv_prune_layers.restype = C.c_int
+    L.sharpv_kv_prune_layers.argtypes = [vp, i64, i64, vp, i64, C.c_int, i32, i32, vp, vp, vp, vp, i64, i64, f32,
+                                         vp, vp, vp, vp, i64, vp, C.POINTER(KVLayout), vp, C.POINTER(KVLayout),
+                                         i32, i32, vp, sz, vp, vp]
     L.sharpv_kv_compact.restype = C.c_int
     L.sharpv_kv_compact.argtypes = [vp, C.POINTER(KVLayout), vp, C.POINTER(KVLayout), i32, i32, vp, vp, i32, i64,
                                     vp, vp]
@@ -336,6 +340,48 @@ def sharpv_kv_compact(kv_src: torch.Tensor, kv_dst: torch.Tensor, kept_pos: torc
         kept_seq_offsets.numel() - 1, capacity, _dev(status_word, "status_word", torch.int32), _stream(stream))
     _check("sharpv_kv_compact", rc)
     return kv_dst
+
+
+def sharpv_kv_prune_layers(hidden_layers: torch.Tensor, visual: torch.Tensor, seq_offsets: torch.Tensor,
+                           vis_begin: torch.Tensor, vis_count: torch.Tensor, vis_offsets: torch.Tensor,
+                           total_seq_tokens: int, kv_src: torch.Tensor, kv_dst: torch.Tensor, M: float = 0.2,
+                           layer_begin: int = 0, capacity: Optional[int] = None, want_mean_cos: bool = False,
+                           workspace=None, status_word=None, stream=None):
+    """Stage two layer by layer.  hidden_layers [n_layers, T, d] holds the hidden states of layers
+    layer_begin .. layer_begin + n_layers - 1.  Returns dict(cos [n, total_visual], kept_pos [n, capacity],
+    kept_seq_offsets [n, B + 1][, mean_cos [n, B]]); kv_dst receives the compacted planes."""
+    if hidden_layers.dim() != 3 or hidden_layers.stride(2) != 1:
+        raise ValueError("hidden_layers must be [layers, tokens, d] with a contiguous last axis")
+    n = hidden_layers.shape[0]
+    ldv = _rows(visual, "visual")
+    if hidden_layers.dtype != visual.dtype or hidden_layers.shape[2] != visual.shape[1]:
+        raise ValueError("hidden_layers and visual must share dtype and feature size")
+    dev = hidden_layers.device
+    B = seq_offsets.numel() - 1
+    total_visual = visual.shape[0]
+    if capacity is None:
+        capacity = total_seq_tokens
+    out = {"cos": torch.empty((n, max(total_visual, 1)), dtype=torch.float32, device=dev),
+           "kept_pos": torch.empty((n, max(capacity, 1)), dtype=torch.int32, device=dev),
+           "kept_seq_offsets": torch.empty((n, B + 1), dtype=torch.int32, device=dev)}
+    if want_mean_cos:
+        out["mean_cos"] = torch.empty((n, B), dtype=torch.float32, device=dev)
+    if total_visual == 0 or capacity == 0:
+        raise ValueError("sharpv_kv_prune_layers wrapper needs total_visual > 0 and capacity > 0")
+    sl, dl = kv_layout(kv_src), kv_layout(kv_dst)
+    ws = _workspace(workspace, sharpv_kv_calibrate_prune_workspace_bytes(total_seq_tokens, B), dev)
+    rc = lib().sharpv_kv_prune_layers(
+        _dev(hidden_layers, "hidden_layers"), hidden_layers.stride(0), hidden_layers.stride(1),
+        _dev(visual, "visual"), ldv, _dtype_code(visual), visual.shape[1], B,
+        _dev(seq_offsets, "seq_offsets", torch.int32), _dev(vis_begin, "vis_begin", torch.int32),
+        _dev(vis_count, "vis_count", torch.int32), _dev(vis_offsets, "vis_offsets", torch.int32),
+        total_seq_tokens, total_visual, float(M), _dev(out["cos"], "cos", torch.float32),
+        _dev(out.get("mean_cos"), "mean_cos", torch.float32), _dev(out["kept_pos"], "kept_pos", torch.int32),
+        _dev(out["kept_seq_offsets"], "kept_seq_offsets", torch.int32), capacity,
+        _dev(kv_src, "kv_src"), C.byref(sl), _dev(kv_dst, "kv_dst"), C.byref(dl), layer_begin, layer_begin + n,
+        ws.data_ptr(), ws.numel(), _dev(status_word, "status_word", torch.int32), _stream(stream))
+    _check("sharpv_kv_prune_layers", rc)
+    return out
 
 
 def sharpv_kv_compact_rope_workspace_bytes(capacity: int, rotary_dim: int) -> int:

@@ -237,6 +237,39 @@ extern "C" sharpv_status sharpv_kv_calibrate_prune(
                           cuda_stream);
 }
 
+// Stage two layer by layer: every layer in the range is calibrated on its own hidden state and only
+// its own K/V planes are compacted with its own kept list (Section 3.2.3 read per layer).
+extern "C" sharpv_status sharpv_kv_prune_layers(
+    const void* hidden, int64_t stride_hidden_layer, int64_t ld_hidden, const void* visual, int64_t ld_visual,
+    sharpv_dtype dtype, int32_t d, int32_t num_seqs, const int32_t* seq_offsets, const int32_t* vis_begin,
+    const int32_t* vis_count, const int32_t* vis_offsets, int64_t total_seq_tokens, int64_t total_visual,
+    float M, float* out_cos, float* out_mean_cos, int32_t* out_kept_pos, int32_t* out_kept_seq_offsets,
+    int64_t capacity, const void* kv_src, const sharpv_kv_layout* src_layout, void* kv_dst,
+    const sharpv_kv_layout* dst_layout, int32_t layer_begin, int32_t layer_end, void* workspace,
+    size_t workspace_bytes, int32_t* status_word, void* cuda_stream) {
+    if (!dtype_ok(dtype)) return SHARPV_ERR_UNSUPPORTED;
+    if (!src_layout || !dst_layout || layer_begin < 0 || layer_begin > layer_end ||
+        layer_end > src_layout->num_layers || stride_hidden_layer < 0 || num_seqs < 1 || capacity < 0)
+        return SHARPV_ERR_INVALID_ARG;
+    if ((stride_hidden_layer * elem_bytes(dtype)) % 16) return SHARPV_ERR_UNSUPPORTED;
+    const int64_t eb = elem_bytes(dtype);
+    for (int32_t l = layer_begin; l < layer_end; ++l) {
+        const int64_t i = l - layer_begin;
+        int32_t* kept_pos = out_kept_pos ? out_kept_pos + i * capacity : nullptr;
+        int32_t* kept_seq_offsets = out_kept_seq_offsets ? out_kept_seq_offsets + i * (num_seqs + 1) : nullptr;
+        sharpv_status st = calibrate_impl(
+            hidden ? (const char*)hidden + i * stride_hidden_layer * eb : nullptr, ld_hidden, visual, ld_visual, dtype,
+            d, num_seqs, seq_offsets, vis_begin, vis_count, vis_offsets, total_seq_tokens, total_visual, M,
+            out_cos ? out_cos + i * total_visual : nullptr, out_mean_cos ? out_mean_cos + i * num_seqs : nullptr,
+            kept_pos, kept_seq_offsets, capacity, workspace, workspace_bytes, status_word, cuda_stream);
+        if (st != SHARPV_OK) return st;
+        st = sharpv_kv_compact(kv_src, src_layout, kv_dst, dst_layout, l, l + 1, kept_pos, kept_seq_offsets, num_seqs,
+                               capacity, status_word, cuda_stream);
+        if (st != SHARPV_OK) return st;
+    }
+    return SHARPV_OK;
+}
+
 // ---------------------------------------------------------------------------------------
 // Allocation-free variant: the scratch lives in a file-scope device array
 // ---------------------------------------------------------------------------------------

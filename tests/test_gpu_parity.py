@@ -318,6 +318,60 @@ def test_layer_wise_reading_of_eq7():
     assert counts[0] > counts[-1] >= wl.n_text
 
 
+def test_layer_by_layer_entry_point():
+    """sharpv_kv_prune_layers (Section 3.2.3 read per layer) against the oracle: per-layer cosines, kept
+    lists and the cache whose layers are compacted with their own lists, in place and into a second cache,
+    for a layer range that starts above layer 0."""
+    L, lb = 5, 1
+    wl = W.custom("layers", 92, W.BF16, 8, 512, 16, [W.make_video_spec(5, 0.9, cuts=[2]), W.make_video_spec(3, 0.8)],
+                  0.0, L, 2, 64)
+    W.fill_tokens(wl)
+    W.fill_kv(wl)
+    T, M = wl.total_seq_tokens, 0.6
+    hidden = []
+    for l in range(lb, L):
+        W.fill_hidden(wl, s_max=0.4 + 0.8 * l)
+        hidden.append(wl.hidden.copy())
+    i32 = lambda a: torch.from_numpy(a).cuda()
+    tabs = [i32(wl.seq_offsets), i32(wl.vis_begin), i32(wl.vis_count), i32(wl.vis_offsets)]
+    d_hidden = torch.stack([to_dev(h) for h in hidden])
+    res, expect = orc.kv_prune_layers(hidden, wl.tokens, wl.seq_offsets, wl.vis_begin, wl.vis_count, wl.vis_offsets,
+                                      M, wl.kv, layer_begin=lb, nthreads=NT)
+    kv = to_dev(wl.kv)
+    g = sv.sharpv_kv_prune_layers(d_hidden, to_dev(wl.tokens), *tabs, T, kv, kv, M=M, layer_begin=lb,
+                                  want_mean_cos=True)
+    torch.cuda.synchronize()
+    exempt = 0
+    for i, o in enumerate(res):
+        assert rel_err(to_host(g["cos"][i]), o["cos"], floor=1.0) <= TIGHT_TOL
+        n = int(g["kept_seq_offsets"][i, -1].item())
+        kept = to_host(g["kept_pos"][i])[:n]
+        sym = np.setxor1d(kept, o["kept_pos"])
+        exempt += sym.size
+        vis_of = {int(p): int(v) for p, v in zip(np.concatenate([wl.seq_offsets[b] + wl.vis_begin[b] + np.arange(wl.vis_count[b])
+                                                                 for b in range(len(wl.vis_count))]),
+                                                 np.concatenate([wl.vis_offsets[b] + np.arange(wl.vis_count[b])
+                                                                 for b in range(len(wl.vis_count))]))}
+        for pos in sym:                     # only tokens whose cosine sits on the threshold may differ
+            assert abs(o["cos"][vis_of[int(pos)]] - M) <= BOUNDARY_TOL
+    assert exempt <= 2
+    if exempt == 0:
+        np.testing.assert_array_equal(to_host(kv), expect)
+        # into a second cache: the prefix of every plane in the range, nothing else
+        dst = torch.zeros_like(kv)
+        g2 = sv.sharpv_kv_prune_layers(d_hidden, to_dev(wl.tokens), *tabs, T, to_dev(wl.kv), dst, M=M, layer_begin=lb)
+        torch.cuda.synchronize()
+        out = to_host(dst)
+        assert np.all(out[:lb] == 0)
+        for i, o in enumerate(res):
+            n = o["kept_pos"].size
+            np.testing.assert_array_equal(out[lb + i][:, :, :n], wl.kv[lb + i][:, :, o["kept_pos"]])
+            assert np.all(out[lb + i][:, :, n:] == 0)
+        np.testing.assert_array_equal(to_host(g2["kept_seq_offsets"]), to_host(g["kept_seq_offsets"]))
+    counts = [int(x) for x in to_host(g["kept_seq_offsets"])[:, -1]]
+    assert counts[0] > counts[-1] >= wl.n_text          # deeper layers keep less
+
+
 def test_kv_compact_one_byte_cache():
     """An fp8-sized cache (one byte per element, 128-byte rows): compaction is a bit copy and needs no
     knowledge of the element format."""

@@ -181,6 +181,33 @@ def test_kv_compact_rope_rejects_bad_arguments(L):
     assert call(lb=1, le=1) == S.OK
 
 
+def test_kv_prune_layers_rejects_bad_arguments(L):
+    def layout(**kw):
+        base = dict(num_layers=4, num_kv_heads=2, head_dim=64, dtype=1, stride_layer=2 * 2 * 500 * 64,
+                    stride_kv=2 * 500 * 64, stride_head=500 * 64, stride_token=64)
+        base.update(kw)
+        return sv.KVLayout(**base)
+
+    def call(hid=P, hs=500 * 512, dtype=1, sl=None, dl=None, lb=0, le=4, B=1, cap=500, ws=P, wsb=1 << 20, kso=P):
+        sl = layout() if sl is None else sl
+        dl = layout() if dl is None else dl
+        return L.sharpv_kv_prune_layers(hid, hs, 512, P, 512, dtype, 512, B, P, P, P, P, 500, 400, 0.2, P, None, P, kso,
+                                        cap, P, C.byref(sl), 2 * P, C.byref(dl), lb, le, ws, wsb, None, None)
+
+    S = sv.Status
+    assert call(lb=2, le=2) == S.OK                               # empty layer range: nothing to do
+    assert call(dtype=7) == S.ERR_UNSUPPORTED
+    assert call(lb=3, le=2) == S.ERR_INVALID_ARG
+    assert call(le=5) == S.ERR_INVALID_ARG                        # beyond the cache's layers
+    assert call(hs=-1) == S.ERR_INVALID_ARG
+    assert call(hs=500 * 512 + 4) == S.ERR_UNSUPPORTED            # layers of hidden states not 16-byte aligned
+    assert call(B=0) == S.ERR_INVALID_ARG
+    assert call(wsb=16) == S.ERR_WORKSPACE                        # from the calibration of the first layer
+    assert call(kso=None) == S.ERR_INVALID_ARG
+    assert L.sharpv_kv_prune_layers(P, 0, 512, P, 512, 1, 512, 1, P, P, P, P, 500, 400, 0.2, P, None, P, P, 500, P,
+                                    None, 2 * P, None, 0, 1, P, 1 << 20, None, None) == S.ERR_INVALID_ARG
+
+
 def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     monkeypatch.setattr(sv, "_lib", None)
     monkeypatch.setattr(sv._build, "LIB_PATH", str(tmp_path / "libsharpv.so"))

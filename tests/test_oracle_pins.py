@@ -394,6 +394,33 @@ def test_kv_compact_is_fancy_indexing():
     np.testing.assert_array_equal(out3, out)
 
 
+def test_layer_by_layer_pruning_is_eq7_per_layer_in_numpy():
+    """The layer-by-layer reading of Eq. 7 (Section 3.2.3) against plain numpy: every layer's kept set is
+    {text} + {visual: cos(h_l, v) >= M} of its own hidden state, and only that layer's planes are compacted."""
+    rng = np.random.default_rng(12)
+    L, H, Dh, d, nv, ntext, M = 3, 2, 8, 16, 10, 3, 0.5
+    T = nv + ntext
+    visual = rng.standard_normal((nv, d)).astype(np.float32)
+    hidden = [np.concatenate([visual + (0.3 + 0.6 * l) * rng.standard_normal((nv, d)).astype(np.float32),
+                              rng.standard_normal((ntext, d)).astype(np.float32)]) for l in range(L)]
+    kv = rng.standard_normal((L + 1, 2, H, T, Dh)).astype(np.float32)
+    so, vb, vc, vo = (np.array(x, np.int32) for x in ([0, T], [0], [nv], [0]))
+    res, out = orc.kv_prune_layers(hidden, visual, so, vb, vc, vo, M, kv, layer_begin=1)
+    np.testing.assert_array_equal(out[0], kv[0])                    # a layer outside the range is untouched
+    sizes = []
+    for l in range(L):
+        h = hidden[l][:nv].astype(np.float64)
+        v = visual.astype(np.float64)
+        cos = (h * v).sum(1) / (np.linalg.norm(h, axis=1) * np.linalg.norm(v, axis=1))
+        np.testing.assert_allclose(res[l]["cos"], cos, rtol=1e-12)
+        kept = np.concatenate([np.nonzero(cos.astype(np.float32) >= np.float32(M))[0], np.arange(nv, T)])
+        np.testing.assert_array_equal(res[l]["kept_pos"], kept)
+        np.testing.assert_array_equal(out[1 + l][:, :, :kept.size], kv[1 + l][:, :, kept])
+        np.testing.assert_array_equal(out[1 + l][:, :, kept.size:], kv[1 + l][:, :, kept.size:])
+        sizes.append(kept.size)
+    assert len(set(sizes)) > 1                                      # the layers really differ
+
+
 def test_kv_compact_inplace_equals_out_of_place_prefix():
     rng = np.random.default_rng(35)
     L, H, T, Dh = 2, 3, 41, 8
