@@ -331,12 +331,21 @@ def run_sharpv(args):
 
     def timed_launches(fn, n):
         """n back-to-back launches between one pair of events (an event pair around a single launch
-        costs several microseconds on its own); returns the mean milliseconds per launch."""
+        costs several microseconds on its own); returns the mean milliseconds per launch.  The n
+        launches (each with its own rotating input copy) are captured into one CUDA graph first, so
+        that the time of the Python caller between two launches is not in the measurement."""
+        g = torch.cuda.CUDAGraph()
+        cs = torch.cuda.Stream()
+        cs.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(cs):
+            with torch.cuda.graph(g, stream=cs):
+                for i in range(n):
+                    fn(i)
+        torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         flush.zero_()
         a.record(stream)
-        for i in range(n):
-            fn(i)
+        g.replay()
         b.record(stream)
         torch.cuda.synchronize()
         return a.elapsed_time(b) / n
