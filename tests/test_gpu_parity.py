@@ -594,6 +594,32 @@ def test_score_random_shapes(seed):
     np.testing.assert_array_equal(to_host(sel["kept_index"])[:off_o[-1]], idx_o)
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("f", [1, 7, 24, 25, 49, 72, 97, 121, 145, 170, 193, 217, 241, 256])
+def test_score_every_frame_size_class(f, bf16):
+    """Frame sizes on both sides of every step in the number of rows a lane keeps in the fused score
+    kernel (one instance of the kernel per step), for both storage types, with a range of tiles that
+    starts inside a video, crosses slices and ends inside a video."""
+    rng = np.random.default_rng(3000 + f)
+    d = 3 * (128 if bf16 else 64)
+    vfo = np.array([0, 4, 4, 9, 11], np.int32)
+    F = int(vfo[-1])
+    x = rng.standard_normal((F * f, d)).astype(np.float32)
+    for t in range(1, F):
+        x[t * f:(t + 1) * f] = 0.95 * x[(t - 1) * f:t * f] + 0.312 * x[t * f:(t + 1) * f]
+    x[6 * f:7 * f] = x[5 * f:6 * f]                 # one exact duplicate frame
+    xs = W.f32_to_bf16_bits(x) if bf16 else x
+    o = orc.score_frames(xs, vfo, f, w=1.0, nthreads=NT)
+    g = sv.sharpv_score_frames(to_dev(xs), torch.from_numpy(vfo).cuda(), F, f, w=1.0, want_spatial=True,
+                               want_temporal=True)
+    torch.cuda.synchronize()
+    for key in ("spatial", "temporal", "importance", "ratio"):
+        e = rel_err(to_host(g[key]), o[key])
+        assert e <= TIGHT_TOL, f"{key}: rel err {e} (f={f}, bf16={bf16})"
+    check_budgets(to_host(g["k"]), o, f)
+    assert np.all(to_host(g["temporal"])[6 * f:7 * f] == 0.0)      # the duplicate frame: exactly zero
+
+
 @pytest.mark.parametrize("seed", range(10))
 def test_stage_two_random_layouts(seed):
     """Random sequence layouts (system tokens before the visual block, sequences without visual tokens,
