@@ -210,6 +210,55 @@ def test_scores_against_numpy_library_routines():
     np.testing.assert_allclose(r["ratio"], np.linalg.norm(T, axis=1) / (2 * math.sqrt(wl.f)), atol=1e-13)
 
 
+# ---------------------------------------------------------------- manual variant (1 - cos), Section 3.1.1
+def test_hand_case_f2_d2_one_minus_cos():
+    """The hand-derived example under the manual variant's dissimilarity: S, T, I and both ratios."""
+    g = _golden("hand_case_f2_d2_one_minus_cos.txt")
+    tokens = np.array([[1, 0], [0, 1], [0, 1], [0, 1]], dtype=np.float32)
+    r = orc.score_frames(tokens, [0, 2], f=2, w=1.0, dissim_kind=orc.ONE_MINUS_COS)
+    S, T, I = r["spatial"], r["temporal"], r["importance"]
+    tol = 1e-14
+    for i, (ks, kt) in enumerate([("S1_0", "T1_0"), ("S1_1", "T1_1"), ("S2_0", "T2_0"), ("S2_1", "T2_1")]):
+        assert abs(S[i] - g[ks]) < tol, (i, S[i])
+        assert abs(T[i] - g[kt]) < tol, (i, T[i])
+    assert abs(I[0] - g["I1_0"]) < tol and abs(I[2] - g["I2_0"]) < tol and abs(I[3] - g["I2_1"]) < tol
+    assert abs(r["ratio"][0] - g["ratio_1"]) < tol and abs(r["ratio"][1] - g["ratio_2"]) < tol
+    assert list(r["k"]) == [0, 0]                                   # floor(0.29), floor(0.71)
+    kn = orc.score_frames(tokens, [0, 2], f=2, dissim_kind=orc.ONE_MINUS_COS, round_mode=orc.ROUND_NEAREST)["k"]
+    assert list(kn) == [0, 1]
+    kc = orc.score_frames(tokens, [0, 2], f=2, dissim_kind=orc.ONE_MINUS_COS, round_mode=orc.ROUND_CEIL)["k"]
+    assert list(kc) == [1, 1]
+
+
+def test_one_minus_cos_scores_against_numpy_and_dissim_identity():
+    """Manual variant on a whole small workload (two videos, so two first frames): S, T, I and the
+    ratio against numpy's 1 - a.b / (|a||b|), and element-wise 1 - cos = Dissim^2 / 2 against the
+    default variant (Eq. 1: Dissim^2 = 2 - 2 cos)."""
+    wl = W.fill_tokens(W.custom("n", 8, W.BF16, 4, 96, 0,
+                                [W.make_video_spec(3, 0.9), W.make_video_spec(2, 0.5)]))
+    x = wl.tokens_as_f32().astype(np.float64).reshape(5, wl.f, wl.d)
+    m = x.mean(axis=1)
+
+    def omc(a, b):
+        return 1.0 - np.sum(a * b, axis=-1) / (np.linalg.norm(a, axis=-1) * np.linalg.norm(b, axis=-1))
+
+    S = np.stack([omc(x[t], m[t][None, :]) for t in range(5)])
+    T = np.stack([S[t] if t in (0, 3) else omc(x[t], x[t - 1]) for t in range(5)])
+    w = 0.7
+    r = orc.score_frames(wl.tokens, wl.video_frame_offsets, wl.f, w=w, dissim_kind=orc.ONE_MINUS_COS)
+    np.testing.assert_allclose(r["spatial"], S.ravel(), atol=1e-12)
+    np.testing.assert_allclose(r["temporal"], T.ravel(), atol=1e-12)
+    np.testing.assert_allclose(r["importance"], (T + w * S).ravel(), atol=1e-12)
+    np.testing.assert_allclose(r["ratio"], np.linalg.norm(T, axis=1) / (2 * math.sqrt(wl.f)), atol=1e-13)
+    # temporal and spatial terms differ on non-first frames, so a swap of kinds in either shows
+    assert np.max(np.abs(T[1] - S[1])) > 1e-3
+    q = orc.score_frames(wl.tokens, wl.video_frame_offsets, wl.f, w=w, dissim_kind=orc.DISSIM)
+    np.testing.assert_allclose(r["spatial"], q["spatial"] ** 2 / 2, atol=1e-14)
+    np.testing.assert_allclose(r["temporal"], q["temporal"] ** 2 / 2, atol=1e-14)
+    # the two kinds really differ (1 - cos != Dissim away from 0 and 2)
+    assert np.max(np.abs(r["temporal"] - q["temporal"])) > 0.1
+
+
 # ---------------------------------------------------------------- statistical closed forms
 def test_statistical_closed_forms_on_generator():
     """Large d, unit-variance tokens: AR(1) rho gives cos ~ rho, T ~ sqrt(2-2rho),
