@@ -8,11 +8,16 @@ score frames -> per-frame top-k + gather -> calibration -> K/V compaction.  Prin
 line (rank 0).  With N > 1 every rank runs the same-shaped batch on its own GPU (videos are
 independent: no data-path collective, weak scaling) and the time is the max over ranks.
 `--impl reference` times the CPU oracle on the host cores instead.
+
+The headline workload is the 256-frame video (the largest single-video configuration; its 2.9 GB
+cache and the destination fit one GPU).  `per_workload` repeats the per-kernel timings on the
+32-frame, 64-frame and ragged-batch configurations in the same run.
 """
 from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import sys
@@ -28,27 +33,38 @@ from paper_2511_08003_b200 import workloads as W  # noqa: E402
 METRIC = "pruning throughput (visual tokens/s)"
 UNIT = "visual tokens/s"
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+MIN_TIMED_SECONDS = 0.3
+KERNEL_REPLAYS = 20
+REPORTED_WORKLOADS = ("onevision_7b", "video_7b", "ragged_batch", "long_video")
+STAGES = ("score", "select", "calibrate", "compact")
 # kernels launched per step by each entry point (score, select, calibrate, compact)
 LAUNCHES_PER_STEP = {"score": 2, "select": 2, "calibrate": 2, "compact": 1}
-# DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/); None = not captured
-NCU_TRAFFIC_BYTES = {("onevision_7b", "compact"): 266_712_320}   # profiles/kv_compact_kernel_onevision_7b.md
+# DRAM read + write bytes of one launch of an entry point's main kernel, from ncu captures.  An entry is
+# used only when the run reproduces the captured launch (same workload, threshold, kept count, plain
+# out-of-place compaction); `commit` is the source revision the counters were taken on.
+NCU_TRAFFIC = {
+    ("onevision_7b", "compact"): {"bytes": 266_712_320, "M": 0.788, "kept_stage_two": 2748, "commit": "ed50430"},
+}
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="onevision_7b", choices=list(W.PRESETS))
+    ap.add_argument("--workload", default="long_video", choices=list(W.PRESETS))
     ap.add_argument("--impl", default="sharpv", choices=["sharpv", "reference"])
     ap.add_argument("--M", type=float, default=0.788,
                     help="degradation threshold; 0.788 keeps about 39 %% of the synthetic visual tokens "
                          "(the paper's reported memory ratio); the paper's default 0.2 keeps all of them")
     ap.add_argument("--w", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--stage", default=None, choices=["score", "select", "calibrate", "compact"],
+    ap.add_argument("--no-per-workload", action="store_true",
+                    help="skip the per-kernel timings of the other configurations")
+    ap.add_argument("--stage", default=None, choices=list(STAGES),
                     help="profiling aid: after the warm-up run only this entry point --steps times "
-                         "(L2 flushed before each) and print its mean duration")
+                         "(HBM-cold inputs) and print its duration")
     ap.add_argument("--inplace", action="store_true",
                     help="compact the K/V cache in place (kv_dst == kv_src) instead of into a second cache")
     ap.add_argument("--rope", action="store_true",
@@ -127,11 +143,31 @@ def host_workload(name, with_kv_layers=None, frames=None, layers=None):
     return wl
 
 
+def oracle_baseline(wl, orc, args, cores, kv_layers, budget_s=25.0):
+    """The oracle as it stands on the host cores: one full pass single-threaded, then full passes on all
+    cores (best kept) while the time budget lasts.  Per stage and in total."""
+    t1, _, _ = oracle_step(wl, orc, args.M, args.w, 1, kv_layers)
+    best, reps, t0 = None, 0, time.perf_counter()
+    while reps < 3 and (reps == 0 or time.perf_counter() - t0 < budget_s):
+        t, _, _ = oracle_step(wl, orc, args.M, args.w, cores, kv_layers)
+        if best is None or sum(t.values()) < sum(best.values()):
+            best = t
+        reps += 1
+    nv = wl.n_visual
+    per_stage = {k: {"s_1_thread": round(t1[k], 4), f"s_{cores}_threads": round(best[k], 4)} for k in t1}
+    return {"value": nv / sum(best.values()), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "single_thread": {"value": nv / sum(t1.values()), "unit": UNIT, "cores": 1},
+            "per_stage": per_stage,
+            "sample": f"the whole workload ({wl.total_frames} frames): one pass on 1 thread, best of {reps} "
+                      f"passes on {cores} OpenMP threads; K/V compaction timed on {kv_layers} of {wl.num_layers} "
+                      f"layers and scaled"}
+
+
 def run_reference(args):
     from oracle import sharpv_oracle as orc
     cores = os.cpu_count() or 1
     kv_layers = 4
-    wl = host_workload(args.workload, with_kv_layers=kv_layers)
+    wl = host_workload(args.workload, with_kv_layers=kv_layers, frames=args.frames)
     for _ in range(min(args.warmup, 1)):
         oracle_step(wl, orc, args.M, args.w, cores, kv_layers)
     t0 = time.perf_counter()
@@ -148,12 +184,19 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "M": args.M, "w": args.w},
+        "config": workload_config(wl, args),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
+
+
+def workload_config(wl, args):
+    """The keys that name the workload; the same on both arms."""
+    return {"workload": args.workload, "frames": wl.total_frames, "tokens_per_frame": wl.f, "d": wl.d,
+            "storage": wl.dtype, "visual_tokens": wl.n_visual, "seq_tokens": wl.total_seq_tokens,
+            "kv": list(wl.kv_shape()), "M": args.M, "w": args.w}
 
 
 # ------------------------------------------------------------------------------------- clocks
@@ -226,7 +269,179 @@ def whole_job_throughput(units_per_rank, world, ms_per_step):
     return world * units_per_rank / (ms_per_step * 1e-3)
 
 
+def replays_per_step(steps, est_step_ms, min_seconds=MIN_TIMED_SECONDS):
+    """How often every timed step is repeated so that the timed region lasts at least min_seconds."""
+    return max(1, int(math.ceil(min_seconds * 1e3 / max(steps * est_step_ms, 1e-9))))
+
+
 # ------------------------------------------------------------------------------------- GPU arm
+class DevicePath:
+    """Device buffers of one workload and the four entry points as callables; nothing is allocated
+    inside a step."""
+
+    L2_BYTES = 126 << 20
+
+    def __init__(self, wl, args, dev, flush):
+        import torch
+        from paper_2511_08003_b200 import binding as sv
+        self.torch, self.sv, self.wl, self.args, self.dev, self.flush = torch, sv, wl, args, dev, flush
+        F, f, d, T, NV = wl.total_frames, wl.f, wl.d, wl.total_seq_tokens, wl.n_visual
+        tdt = torch.float32 if wl.dtype == W.F32 else torch.bfloat16
+
+        def dev_tokens(a):
+            if a.dtype == np.uint16:
+                return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+            return torch.from_numpy(a).to(dev)
+
+        # Rotating copies of the token and hidden-state matrices: consecutive launches of one kernel
+        # read different copies, and a copy is only read again after more than twice the L2 capacity of
+        # other data has gone through the cache, so every timed launch starts from HBM.
+        in_bytes = wl.tokens.nbytes
+        self.ncopies = max(1, -(-2 * self.L2_BYTES // in_bytes) + 1) if in_bytes < 2 * self.L2_BYTES else 1
+        self.tok_copies = [dev_tokens(wl.tokens) for _ in range(self.ncopies)]
+        self.hid_copies = [dev_tokens(wl.hidden) for _ in range(self.ncopies)]
+        self.tokens, self.hidden = self.tok_copies[0], self.hid_copies[0]
+        self.tabs = {k: torch.from_numpy(getattr(wl, k)).to(dev) for k in
+                     ("video_frame_offsets", "seq_offsets", "vis_begin", "vis_count", "vis_offsets")}
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(wl.seed * 1000 + 3)
+        self.kv = torch.empty(wl.kv_shape(), dtype=tdt, device=dev)
+        for l in range(wl.num_layers):                  # N(0,1) K/V, drawn on the device layer by layer
+            self.kv[l] = torch.randn(wl.kv_shape()[1:], dtype=torch.float32, device=dev, generator=gen).to(tdt)
+        self.kv_dst = self.kv if args.inplace else torch.zeros_like(self.kv)
+
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.o_score = {"importance": torch.empty(NV, dtype=torch.float32, device=dev),
+                        "ratio": torch.empty(F, dtype=torch.float32, device=dev),
+                        "k": torch.empty(F, dtype=torch.int32, device=dev)}
+        self.ws_score = torch.empty(sv.sharpv_score_frames_workspace_bytes(F, f, d), dtype=torch.uint8, device=dev)
+        self.o_sel = {"kept_index": torch.empty(NV, dtype=torch.int32, device=dev),
+                      "kept_offsets": torch.empty(F + 1, dtype=torch.int32, device=dev),
+                      "num_kept": torch.empty(1, dtype=torch.int32, device=dev),
+                      "tokens": torch.empty((NV, d), dtype=tdt, device=dev)}
+        self.ws_sel = torch.empty(sv.sharpv_select_tokens_workspace_bytes(F, f), dtype=torch.uint8, device=dev)
+        self.o_cal = {"cos": torch.empty(NV, dtype=torch.float32, device=dev),
+                      "kept_pos": torch.empty(T, dtype=torch.int32, device=dev),
+                      "kept_seq_offsets": torch.empty(wl.num_videos + 1, dtype=torch.int32, device=dev)}
+        self.ws_cal = torch.empty(sv.sharpv_kv_calibrate_prune_workspace_bytes(T, wl.num_videos), dtype=torch.uint8,
+                                  device=dev)
+        self.ws_rope = (torch.empty(sv.sharpv_kv_compact_rope_workspace_bytes(T, wl.head_dim), dtype=torch.uint8,
+                                    device=dev) if args.rope else None)
+        self.stages = {"score": self.stage_score, "select": self.stage_select, "calibrate": self.stage_calibrate,
+                       "compact": self.stage_compact}
+        self.n_keep = self.t_keep = None
+
+    def stage_score(self, i=0):
+        wl = self.wl
+        self.sv.sharpv_score_frames(self.tok_copies[i % self.ncopies], self.tabs["video_frame_offsets"],
+                                    wl.total_frames, wl.f, w=self.args.w, out=self.o_score, workspace=self.ws_score,
+                                    status_word=self.status)
+
+    def stage_select(self, i=0):
+        wl = self.wl
+        self.sv.sharpv_select_tokens(self.o_score["importance"], self.o_score["k"], wl.total_frames, wl.f,
+                                     tokens=self.tok_copies[i % self.ncopies], capacity=wl.n_visual, out=self.o_sel,
+                                     workspace=self.ws_sel, status_word=self.status)
+
+    def stage_calibrate(self, i=0):
+        wl, t = self.wl, self.tabs
+        self.sv.sharpv_kv_calibrate_prune(self.hid_copies[i % self.ncopies], self.tok_copies[i % self.ncopies],
+                                          t["seq_offsets"], t["vis_begin"], t["vis_count"], t["vis_offsets"],
+                                          wl.total_seq_tokens, M=self.args.M, capacity=wl.total_seq_tokens,
+                                          out=self.o_cal, workspace=self.ws_cal, status_word=self.status)
+
+    def stage_compact(self, i=0):
+        wl = self.wl
+        T = wl.total_seq_tokens
+        if self.args.rope:
+            self.sv.sharpv_kv_compact_rope(self.kv, self.kv_dst, self.o_cal["kept_pos"], self.o_cal["kept_seq_offsets"],
+                                           self.tabs["seq_offsets"], T, wl.head_dim, 1.0e6, workspace=self.ws_rope,
+                                           status_word=self.status)
+            return
+        self.sv.sharpv_kv_compact(self.kv, self.kv_dst, self.o_cal["kept_pos"], self.o_cal["kept_seq_offsets"],
+                                  capacity=T, status_word=self.status)
+
+    def step(self):
+        for name in STAGES:
+            self.stages[name]()
+
+    def warm(self, n):
+        torch = self.torch
+        for _ in range(n):
+            self.flush.zero_()
+            self.step()
+        torch.cuda.synchronize()
+        self.n_keep = int(self.o_sel["num_kept"].item())
+        self.t_keep = int(self.o_cal["kept_seq_offsets"][-1].item())
+        assert int(self.status.item()) == 0, "device status word set"
+
+    def capture(self, fn):
+        torch = self.torch
+        g = torch.cuda.CUDAGraph()
+        cs = torch.cuda.Stream()
+        cs.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(cs):
+            with torch.cuda.graph(g, stream=cs):
+                fn()
+        torch.cuda.synchronize()
+        return g
+
+    def time_stage(self, name, replays=KERNEL_REPLAYS, inner=None):
+        """Launch durations of one entry point from HBM-cold inputs.  `inner` back-to-back launches, each
+        on its own rotating input copy, are captured into one CUDA graph (an event pair around a single
+        launch costs several microseconds on its own, and the Python caller's time between two launches
+        must not be measured); the graph is replayed `replays` times, each replay between its own pair of
+        events on the launching stream.  Returns per-launch milliseconds: median, best and mean over the
+        replays."""
+        torch = self.torch
+        fn = self.stages[name]
+        stream = torch.cuda.current_stream()
+
+        def graph_of(n):
+            return self.capture(lambda: [fn(i) for i in range(n)])
+
+        if inner is None:
+            g = graph_of(self.ncopies)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            self.flush.zero_()
+            a.record(stream)
+            g.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            est_ms = a.elapsed_time(b) / self.ncopies
+            # a replay should last about half a millisecond, and walk through all input copies
+            inner = min(64, max(self.ncopies, int(math.ceil(0.5 / max(est_ms, 1e-4)))))
+            inner = -(-inner // self.ncopies) * self.ncopies
+        g = graph_of(inner)
+        per_launch = []
+        self.flush.zero_()
+        g.replay()                                          # one untimed replay
+        for _ in range(replays):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            g.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            per_launch.append(a.elapsed_time(b) / inner)
+        return {"median_ms": statistics.median(per_launch), "best_ms": min(per_launch),
+                "mean_ms": statistics.fmean(per_launch), "replays": replays, "launches_per_replay": inner}
+
+    def kernel_table(self, peak):
+        out = {}
+        for name in STAGES:
+            t = self.time_stage(name)
+            b = algorithmic_bytes(self.wl, self.n_keep, self.t_keep, name)
+            gbs = b / (t["median_ms"] * 1e-3) / 1e9
+            out[name] = {"ms": round(t["median_ms"], 5), "median_ms": round(t["median_ms"], 5),
+                         "best_ms": round(t["best_ms"], 5), "algorithmic_bytes": b, "GBps": round(gbs, 1),
+                         "frac": round(gbs / peak, 4), "frac_of_measured": round(gbs / peak, 4),
+                         "frac_of_nominal_8000": round(gbs / NOMINAL_HBM_GBS, 4),
+                         "best_GBps": round(b / (t["best_ms"] * 1e-3) / 1e9, 1),
+                         "launches": LAUNCHES_PER_STEP[name], "replays": t["replays"],
+                         "launches_per_replay": t["launches_per_replay"]}
+        return out
+
+
 def run_sharpv(args):
     import torch
     import torch.distributed as dist
@@ -242,86 +457,11 @@ def run_sharpv(args):
     dev = torch.device("cuda", local_rank)
     sv.lib()                                            # fail loudly before any work if not built
 
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)      # > 2x the 126 MB L2
     wl = host_workload(args.workload, frames=args.frames, layers=args.layers)
     F, f, d, T, NV = wl.total_frames, wl.f, wl.d, wl.total_seq_tokens, wl.n_visual
-    tdt = torch.float32 if wl.dtype == W.F32 else torch.bfloat16
-
-    def dev_tokens(a):
-        if a.dtype == np.uint16:
-            return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
-        return torch.from_numpy(a).to(dev)
-
-    def pinned(a):
-        t = torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
-        return t.view(torch.bfloat16) if a.dtype == np.uint16 else t
-
-    # Rotating copies of the token and hidden-state matrices: consecutive launches of one kernel
-    # read different copies, and a copy is only read again after more than twice the L2 capacity of
-    # other data has gone through the cache, so every timed launch starts from HBM.
-    L2_BYTES = 126 << 20
-    in_bytes = wl.tokens.nbytes
-    ncopies = max(1, -(-2 * L2_BYTES // in_bytes) + 1) if in_bytes < 2 * L2_BYTES else 1
-    tok_copies = [dev_tokens(wl.tokens) for _ in range(ncopies)]
-    hid_copies = [dev_tokens(wl.hidden) for _ in range(ncopies)]
-    tokens, hidden = tok_copies[0], hid_copies[0]
-    tabs = {k: torch.from_numpy(getattr(wl, k)).to(dev) for k in
-            ("video_frame_offsets", "seq_offsets", "vis_begin", "vis_count", "vis_offsets")}
-    gen = torch.Generator(device=dev)
-    gen.manual_seed(wl.seed * 1000 + 3)
-    kv = torch.empty(wl.kv_shape(), dtype=tdt, device=dev)
-    for l in range(wl.num_layers):                      # N(0,1) K/V, drawn on the device layer by layer
-        kv[l] = torch.randn(wl.kv_shape()[1:], dtype=torch.float32, device=dev, generator=gen).to(tdt)
-    kv_dst = torch.zeros_like(kv)
-
-    # preallocated outputs and workspaces: nothing is allocated inside a step
-    status = torch.zeros(1, dtype=torch.int32, device=dev)
-    o_score = {"importance": torch.empty(NV, dtype=torch.float32, device=dev),
-               "ratio": torch.empty(F, dtype=torch.float32, device=dev),
-               "k": torch.empty(F, dtype=torch.int32, device=dev)}
-    ws_score = torch.empty(sv.sharpv_score_frames_workspace_bytes(F, f, d), dtype=torch.uint8, device=dev)
-    o_sel = {"kept_index": torch.empty(NV, dtype=torch.int32, device=dev),
-             "kept_offsets": torch.empty(F + 1, dtype=torch.int32, device=dev),
-             "num_kept": torch.empty(1, dtype=torch.int32, device=dev),
-             "tokens": torch.empty((NV, d), dtype=tdt, device=dev)}
-    ws_sel = torch.empty(sv.sharpv_select_tokens_workspace_bytes(F, f), dtype=torch.uint8, device=dev)
-    o_cal = {"cos": torch.empty(NV, dtype=torch.float32, device=dev),
-             "kept_pos": torch.empty(T, dtype=torch.int32, device=dev),
-             "kept_seq_offsets": torch.empty(wl.num_videos + 1, dtype=torch.int32, device=dev)}
-    ws_cal = torch.empty(sv.sharpv_kv_calibrate_prune_workspace_bytes(T, wl.num_videos), dtype=torch.uint8,
-                         device=dev)
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)      # > 2x the 126 MB L2
+    path = DevicePath(wl, args, dev, flush)
     stream = torch.cuda.current_stream()
-
-    def stage_score(i=0):
-        sv.sharpv_score_frames(tok_copies[i % ncopies], tabs["video_frame_offsets"], F, f, w=args.w, out=o_score,
-                               workspace=ws_score, status_word=status)
-
-    def stage_select(i=0):
-        sv.sharpv_select_tokens(o_score["importance"], o_score["k"], F, f, tokens=tok_copies[i % ncopies],
-                                capacity=NV, out=o_sel, workspace=ws_sel, status_word=status)
-
-    def stage_calibrate(i=0):
-        sv.sharpv_kv_calibrate_prune(hid_copies[i % ncopies], tok_copies[i % ncopies], tabs["seq_offsets"],
-                                     tabs["vis_begin"], tabs["vis_count"], tabs["vis_offsets"], T, M=args.M,
-                                     capacity=T, out=o_cal, workspace=ws_cal, status_word=status)
-
-    ws_rope = (torch.empty(sv.sharpv_kv_compact_rope_workspace_bytes(T, wl.head_dim), dtype=torch.uint8, device=dev)
-               if args.rope else None)
-
-    def stage_compact(i=0):
-        if args.rope:
-            sv.sharpv_kv_compact_rope(kv, kv_dst, o_cal["kept_pos"], o_cal["kept_seq_offsets"], tabs["seq_offsets"],
-                                      T, wl.head_dim, 1.0e6, workspace=ws_rope, status_word=status)
-            return
-        sv.sharpv_kv_compact(kv, kv if args.inplace else kv_dst, o_cal["kept_pos"], o_cal["kept_seq_offsets"],
-                             capacity=T, status_word=status)
-
-    stages = [("score", stage_score), ("select", stage_select), ("calibrate", stage_calibrate),
-              ("compact", stage_compact)]
-
-    def step():
-        for _, fn in stages:
-            fn()
 
     def barrier():
         torch.cuda.synchronize()
@@ -329,59 +469,40 @@ def run_sharpv(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed_launches(fn, n):
-        """n back-to-back launches between one pair of events (an event pair around a single launch
-        costs several microseconds on its own); returns the mean milliseconds per launch.  The n
-        launches (each with its own rotating input copy) are captured into one CUDA graph first, so
-        that the time of the Python caller between two launches is not in the measurement."""
-        g = torch.cuda.CUDAGraph()
-        cs = torch.cuda.Stream()
-        cs.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(cs):
-            with torch.cuda.graph(g, stream=cs):
-                for i in range(n):
-                    fn(i)
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        flush.zero_()
-        a.record(stream)
-        g.replay()
-        b.record(stream)
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / n
-
     W_ = max(args.warmup, 3)
-    for _ in range(W_):
-        flush.zero_()
-        step()
-    torch.cuda.synchronize()
-    n_keep = int(o_sel["num_kept"].item())
-    t_keep = int(o_cal["kept_seq_offsets"][-1].item())
-    assert int(status.item()) == 0, "device status word set"
+    path.warm(W_)
+    n_keep, t_keep = path.n_keep, path.t_keep
 
     if args.stage:
-        fn = dict(stages)[args.stage]
-        ms = timed_launches(fn, args.steps)
+        t = path.time_stage(args.stage, replays=max(3, min(args.steps, KERNEL_REPLAYS)),
+                            inner=path.ncopies if args.steps <= 3 else None)
         nbytes = algorithmic_bytes(wl, n_keep, t_keep, args.stage)
-        print(json.dumps({"stage": args.stage, "workload": args.workload, "frames": F, "ms": ms,
-                          "algorithmic_bytes": nbytes, "GBps": nbytes / (ms * 1e-3) / 1e9,
-                          "kept_stage_one": n_keep, "kept_stage_two": t_keep, "input_copies": ncopies}))
+        print(json.dumps({"stage": args.stage, "workload": args.workload, "frames": F, "ms": t["median_ms"],
+                          "best_ms": t["best_ms"], "algorithmic_bytes": nbytes,
+                          "GBps": nbytes / (t["median_ms"] * 1e-3) / 1e9, "kept_stage_one": n_keep,
+                          "kept_stage_two": t_keep, "input_copies": path.ncopies,
+                          "launches_per_replay": t["launches_per_replay"], "replays": t["replays"]}))
         return
 
     # The library calls only enqueue kernels (no allocation, no sync), so one step is captured
     # into a CUDA graph and replayed: the GPU never waits for the Python caller.
-    graph = torch.cuda.CUDAGraph()
-    cap_stream = torch.cuda.Stream()
-    cap_stream.wait_stream(torch.cuda.current_stream())
-    with torch.cuda.stream(cap_stream):
-        with torch.cuda.graph(graph, stream=cap_stream):
-            step()
-    torch.cuda.synchronize()
+    graph = path.capture(path.step)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
     for _ in range(W_):
         graph.replay()
+    e1.record(stream)
     torch.cuda.synchronize()
+    est_step_ms = e0.elapsed_time(e1) / W_
+    # every timed step is repeated until the timed region lasts MIN_TIMED_SECONDS, whatever --steps is
+    inner = replays_per_step(args.steps, est_step_ms)
+    if world > 1:
+        t = torch.tensor([inner], dtype=torch.int64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        inner = int(t.item())
+    replays = args.steps * inner
 
-    # ---- timed region: K graph replays back to back between one pair of events.  A step reads and
+    # ---- timed region: back-to-back graph replays between one pair of events.  A step reads and
     # writes several times the L2 capacity, so each step finds its inputs in HBM, not in cache.
     try:
         pr = torch.cuda.get_device_properties(dev)
@@ -394,7 +515,7 @@ def run_sharpv(args):
     barrier()
     wall0 = time.perf_counter()
     e0.record(stream)
-    for _ in range(args.steps):
+    for _ in range(replays):
         graph.replay()
     e1.record(stream)
     barrier()
@@ -402,19 +523,19 @@ def run_sharpv(args):
     total_ms = e0.elapsed_time(e1)
 
     # ---- per-entry-point launch durations from HBM-cold inputs, in the same region of the run
-    stage_n = max(10, min(args.steps, 100))
-    stage_ms = {name: timed_launches(fn, stage_n) for name, fn in stages}
+    peak, peak_kind = measured_peak()
+    kernels = path.kernel_table(peak)
 
     # ---- secondary number: stage two chained behind stage one (it sees only the tokens stage one kept).
     # The survivors' features, hidden rows and K/V rows are laid out once with torch indexing (set-up,
     # not timed); calibration and compaction then run on that smaller sequence set.
     chained = None
-    if world == 1 and wl.num_videos == 1 and n_keep > 0:
-        idx = o_sel["kept_index"][:n_keep].long()
+    if world == 1 and wl.num_videos == 1 and n_keep > 0 and not args.inplace and not args.rope:
+        idx = path.o_sel["kept_index"][:n_keep].long()
         pos = torch.cat([idx, torch.arange(NV, T, device=dev)])            # survivors, then the text tokens
-        c_vis = tokens.index_select(0, idx).contiguous()
-        c_hid = hidden.index_select(0, pos).contiguous()
-        c_kv = kv.index_select(3, pos).contiguous()
+        c_vis = path.tokens.index_select(0, idx).contiguous()
+        c_hid = path.hidden.index_select(0, pos).contiguous()
+        c_kv = path.kv.index_select(3, pos).contiguous()
         c_dst = torch.zeros_like(c_kv)
         Tc = int(pos.numel())
         i32 = lambda v: torch.tensor(v, dtype=torch.int32, device=dev)
@@ -426,15 +547,16 @@ def run_sharpv(args):
 
         def chained_stage_two(i=0):
             sv.sharpv_kv_calibrate_prune(c_hid, c_vis, *c_tabs, Tc, M=args.M, capacity=Tc, out=c_out,
-                                         workspace=c_ws, status_word=status)
+                                         workspace=c_ws, status_word=path.status)
             sv.sharpv_kv_compact(c_kv, c_dst, c_out["kept_pos"], c_out["kept_seq_offsets"], capacity=Tc,
-                                 status_word=status)
+                                 status_word=path.status)
 
         chained_stage_two()
         torch.cuda.synchronize()
-        c_ms = timed_launches(chained_stage_two, stage_n)
+        path.stages["chained"] = chained_stage_two
+        c_t = path.time_stage("chained", replays=10, inner=4)
         c_keep = int(c_out["kept_seq_offsets"][-1].item())
-        chained = {"seq_tokens": Tc, "kept_stage_two": c_keep, "stage_two_ms": round(c_ms, 5),
+        chained = {"seq_tokens": Tc, "kept_stage_two": c_keep, "stage_two_ms": round(c_t["median_ms"], 5),
                    "token_budget": round((c_keep - (T - NV)) / NV, 4),
                    "note": "calibration + compaction on the survivors of stage one; token_budget = visual "
                            "tokens left after both stages / visual tokens in"}
@@ -442,10 +564,14 @@ def run_sharpv(args):
     clocks = sampler.stop() if sampler else None
 
     total_ms = max_over_ranks(total_ms, dev, world)
-    ms_per_step = total_ms / args.steps
+    ms_per_step = total_ms / replays
     value = whole_job_throughput(NV, world, ms_per_step)
 
     # ---- end to end: inputs start in pinned host memory, results are read back every step
+    def pinned(a):
+        t = torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+        return t.view(torch.bfloat16) if a.dtype == np.uint16 else t
+
     h_tokens, h_hidden = pinned(wl.tokens), pinned(wl.hidden)
     h_idx = torch.empty(NV, dtype=torch.int32).pin_memory()
     h_pos = torch.empty(T, dtype=torch.int32).pin_memory()
@@ -453,13 +579,13 @@ def run_sharpv(args):
     h_kso = torch.empty(wl.num_videos + 1, dtype=torch.int32).pin_memory()
 
     def e2e_step():
-        tokens.copy_(h_tokens, non_blocking=True)
-        hidden.copy_(h_hidden, non_blocking=True)
-        step()
-        h_idx.copy_(o_sel["kept_index"], non_blocking=True)
-        h_cnt.copy_(o_sel["kept_offsets"], non_blocking=True)
-        h_pos.copy_(o_cal["kept_pos"], non_blocking=True)
-        h_kso.copy_(o_cal["kept_seq_offsets"], non_blocking=True)
+        path.tokens.copy_(h_tokens, non_blocking=True)
+        path.hidden.copy_(h_hidden, non_blocking=True)
+        path.step()
+        h_idx.copy_(path.o_sel["kept_index"], non_blocking=True)
+        h_cnt.copy_(path.o_sel["kept_offsets"], non_blocking=True)
+        h_pos.copy_(path.o_cal["kept_pos"], non_blocking=True)
+        h_kso.copy_(path.o_cal["kept_seq_offsets"], non_blocking=True)
         torch.cuda.synchronize()
 
     e2e_steps = max(3, min(args.steps, 10))
@@ -482,55 +608,72 @@ def run_sharpv(args):
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = measured_peak()
-    kernels = {}
-    for name, _ in stages:
-        b = algorithmic_bytes(wl, n_keep, t_keep, name)
-        gbs = b / (stage_ms[name] * 1e-3) / 1e9
-        kernels[name] = {"ms": round(stage_ms[name], 5), "algorithmic_bytes": b, "GBps": round(gbs, 1),
-                         "frac": round(gbs / peak, 4), "launches": LAUNCHES_PER_STEP[name]}
-    dom = max(stage_ms, key=stage_ms.get)
+    dom = max(STAGES, key=lambda k: kernels[k]["median_ms"])
+    cap = NCU_TRAFFIC.get((args.workload, dom))
+    same_launch = (cap is not None and not args.inplace and not args.rope and args.frames is None and
+                   args.layers is None and abs(cap["M"] - args.M) < 1e-9 and cap["kept_stage_two"] == t_keep)
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["GBps"], "peak": peak, "unit": "GB/s",
                 "frac": kernels[dom]["frac"], "peak_source": f"of {peak_kind}",
-                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dom))}
+                "frac_of_nominal_8000": kernels[dom]["frac_of_nominal_8000"],
+                "achieved_basis": "algorithmic bytes of one launch / median launch duration (CUDA events)",
+                "traffic": cap["bytes"] if same_launch else None,
+                "traffic_commit": cap["commit"] if same_launch else None}
+
+    # ---- the same per-kernel timings on the other configurations (HBM-cold, same method)
+    per_workload = {args.workload: {k: {x: kernels[k][x] for x in
+                                        ("median_ms", "best_ms", "GBps", "frac_of_measured", "frac_of_nominal_8000")}
+                                    for k in STAGES}}
+    per_workload[args.workload]["frames"] = F
+    if world == 1 and not args.no_per_workload and args.frames is None and args.layers is None:
+        del path, graph
+        torch.cuda.empty_cache()
+        for name in REPORTED_WORKLOADS:
+            if name in per_workload:
+                continue
+            owl = host_workload(name)
+            op = DevicePath(owl, args, dev, flush)
+            op.warm(3)
+            tab = op.kernel_table(peak)
+            per_workload[name] = {k: {x: tab[k][x] for x in
+                                      ("median_ms", "best_ms", "GBps", "frac_of_measured", "frac_of_nominal_8000")}
+                                  for k in STAGES}
+            per_workload[name]["frames"] = owl.total_frames
+            per_workload[name]["kept_stage_one"] = op.n_keep
+            per_workload[name]["kept_stage_two"] = op.t_keep
+            del op, owl
+            torch.cuda.empty_cache()
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:
         from oracle import sharpv_oracle as orc
         cores = os.cpu_count() or 1
         kv_layers = 2
-        hw = host_workload(args.workload, with_kv_layers=kv_layers)
-        best = None
-        t0 = time.perf_counter()
-        reps = 0
-        while reps < 3 and time.perf_counter() - t0 < 25:
-            t, _, _ = oracle_step(hw, orc, args.M, args.w, cores, kv_layers)
-            tot = sum(t.values())
-            best = tot if best is None else min(best, tot)
-            reps += 1
-        cpu = {"value": NV / best, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"best of {reps} full passes of the same workload (K/V compaction timed on {kv_layers} of "
-                         f"{wl.num_layers} layers and scaled), {cores} OpenMP threads"}
+        hw = host_workload(args.workload, with_kv_layers=kv_layers, frames=args.frames)
+        cpu = oracle_baseline(hw, orc, args, cores, kv_layers)
 
+    cfg = workload_config(wl, args)
+    cfg.update({"kept_stage_one": n_keep, "kept_stage_two": t_keep, "kv_in_place": bool(args.inplace),
+                "kv_rope": bool(args.rope),
+                "launch": f"one CUDA graph replay per pass; every timed step = {inner} passes back to back, so that "
+                          f"the timed region lasts at least {MIN_TIMED_SECONDS} s",
+                "l2": "inputs larger than L2: a step streams several times the 126 MB L2 (K/V alone is "
+                      "larger), and the per-kernel timings rotate through input copies totalling more than "
+                      "twice the L2"})
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": W_, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": W_, "ms_per_step": ms_per_step, "replays": replays, "replays_per_step": inner,
+        "timed_region_s": round(total_ms * 1e-3, 4), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": args.workload, "frames": F, "tokens_per_frame": f, "d": d, "storage": wl.dtype,
-                   "visual_tokens": NV, "seq_tokens": T, "kv": list(wl.kv_shape()), "M": args.M, "w": args.w,
-                   "kept_stage_one": n_keep, "kept_stage_two": t_keep, "kv_in_place": bool(args.inplace), "kv_rope": bool(args.rope),
-                   "launch": "one CUDA graph replay per step, steps back to back",
-                   "l2": "inputs larger than L2: a step streams several times the 126 MB L2 (K/V alone is "
-                         "larger), and the per-kernel timings rotate through input copies totalling more than "
-                         "twice the L2"},
+        "config": cfg,
         "kv_compaction_GBps": kernels["compact"]["GBps"], "chained": chained,
-        "roofline": roofline, "kernels": kernels,
+        "roofline": roofline, "kernels": kernels, "per_workload": per_workload,
+        "peaks": {"hbm_measured_GBps": peak, "hbm_nominal_GBps": NOMINAL_HBM_GBS, "source": peak_kind},
         "cpu_baseline": cpu,
         "e2e": {"value": whole_job_throughput(NV, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "note": "tokens and hidden state copied from pinned host memory every step, kept-index lists "
                         "read back; the K/V cache is device-resident model state"},
-        "gpu_launches": sum(LAUNCHES_PER_STEP.values()) * args.steps,
+        "gpu_launches": sum(LAUNCHES_PER_STEP.values()) * replays,
         "clocks": clocks, "wall_s": round(wall, 3),
     }
     print(json.dumps(line))

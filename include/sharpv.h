@@ -217,7 +217,9 @@ sharpv_status sharpv_kv_calibrate_prune_noalloc(
  * multiple of 16 bytes; a row (head_dim elements) may be at most 16 KB.  The benchmarked layout is
  * [L][2][H][T][D_h]; a token-major cache is expressed through the strides.  kv_dst == kv_src with identical strides compacts in place (every
  * plane is walked front to back; serving stacks that cannot afford a second cache use this);
- * otherwise dst must not overlap src.  Rows of dst at and beyond
+ * otherwise dst must not overlap src: the byte ranges that the first `capacity` token rows of the planes of
+ * [layer_begin, layer_end) span in the two caches must be disjoint, or SHARPV_ERR_INVALID_ARG is returned and
+ * nothing is launched.  Rows of dst at and beyond
  * n_kept are left untouched.  `capacity` is an upper bound on n_kept that the host knows
  * (for example total_seq_tokens) and sizes the launch; rows beyond it are not copied.
  */

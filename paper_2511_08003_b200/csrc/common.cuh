@@ -21,6 +21,28 @@ inline bool dtype_ok(sharpv_dtype dt) { return dt == SHARPV_F32 || dt == SHARPV_
 inline bool copy_dtype_ok(sharpv_dtype dt) { return dtype_ok(dt) || dt == SHARPV_U8; }    // bit copies only
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Byte range [lo, hi) that the first `rows` token rows of every plane of the layers
+// [layer_begin, layer_end) can touch (strides are non-negative, so the range starts at the first
+// layer's K block and ends behind the last row of the last layer's last V head).
+inline void kv_extent(const void* base, const sharpv_kv_layout* L, int layer_begin, int layer_end, int64_t rows,
+                      uintptr_t& lo, uintptr_t& hi) {
+    const int64_t eb = elem_bytes(L->dtype);
+    lo = reinterpret_cast<uintptr_t>(base) + (uintptr_t)(layer_begin * L->stride_layer * eb);
+    hi = reinterpret_cast<uintptr_t>(base) +
+         (uintptr_t)(((layer_end - 1) * L->stride_layer + L->stride_kv + (L->num_kv_heads - 1) * L->stride_head +
+                      (rows - 1) * L->stride_token + L->head_dim) * eb);
+}
+
+// true when the first `rows` rows of the planes of [layer_begin, layer_end) of two caches share bytes
+inline bool kv_ranges_overlap(const void* a, const sharpv_kv_layout* la, const void* b, const sharpv_kv_layout* lb,
+                              int layer_begin, int layer_end, int64_t rows) {
+    if (layer_end <= layer_begin || rows <= 0) return false;
+    uintptr_t a_lo, a_hi, b_lo, b_hi;
+    kv_extent(a, la, layer_begin, layer_end, rows, a_lo, a_hi);
+    kv_extent(b, lb, layer_begin, layer_end, rows, b_lo, b_hi);
+    return a_lo < b_hi && b_lo < a_hi;
+}
+
 inline sharpv_status launch_status() {
     return cudaGetLastError() == cudaSuccess ? SHARPV_OK : SHARPV_ERR_CUDA;
 }

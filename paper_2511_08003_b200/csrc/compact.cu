@@ -170,6 +170,12 @@ extern "C" sharpv_status sharpv_kv_compact(
     const int planes = (layer_end - layer_begin) * 2 * src_layout->num_kv_heads;
     if (planes == 0 || capacity == 0) return SHARPV_OK;
     if (planes > 65535) return SHARPV_ERR_UNSUPPORTED;
+    if (!in_place) {
+        // a destination that shares bytes with the source without being the source itself would be
+        // overwritten while other CTAs still read it
+        if (kv_ranges_overlap(kv_src, src_layout, kv_dst, dst_layout, layer_begin, layer_end, capacity))
+            return SHARPV_ERR_INVALID_ARG;
+    }
 
     const int64_t eb = elem_bytes(src_layout->dtype);
     PlaneGeom g;

@@ -190,6 +190,8 @@ extern "C" sharpv_status sharpv_kv_compact_rope(
     if (capacity >= (int64_t)1 << 31) return SHARPV_ERR_UNSUPPORTED;
     const int planes = (layer_end - layer_begin) * 2 * src_layout->num_kv_heads;
     if (planes == 0 || capacity == 0) return SHARPV_OK;
+    if (kv_ranges_overlap(kv_src, src_layout, kv_dst, dst_layout, layer_begin, layer_end, capacity))
+        return SHARPV_ERR_INVALID_ARG;
     if (rotary_dim > 0 && (!workspace || !aligned16(workspace))) return SHARPV_ERR_INVALID_ARG;
     if (workspace_bytes < sharpv_kv_compact_rope_workspace_bytes(capacity, rotary_dim)) return SHARPV_ERR_WORKSPACE;
 

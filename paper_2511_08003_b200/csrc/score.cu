@@ -1,7 +1,7 @@
 // Stage one (a): spatial / temporal dissimilarity scores and the adaptive per-frame budget
 // (Section 3.1.2 - 3.1.3, Eq. 1-6).
 //
-// Shapes that split into 256-byte column slices with frames of up to 256 tokens run in the single
+// Shapes that split into 128-byte column slices with frames of up to 256 tokens run in the single
 // fused kernel of score_fused.cu.  Every other shape runs the three kernels below:
 //   frame_mean_kernel   column sums of each frame -> frame mean (fp32), first-frame flags
 //   row_scores_kernel   one warp per token: the row reductions behind S, T and I

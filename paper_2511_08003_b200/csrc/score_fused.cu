@@ -1,24 +1,24 @@
 // Stage one (a) with one HBM read per token (Section 3.1.2 - 3.1.3, Eq. 1-6).
 //
-// The token matrix is cut into column slices of 256 bytes.  A work unit is (slice s, frame t):
-// the f x 256-byte tile of frame t.  Persistent CTAs (one per SM) each take a contiguous range of
-// units in (slice-major, frame-minor) order, so a CTA walks consecutive frames of one slice.
+// The token matrix is cut into column slices of 128 bytes.  A work unit is (slice s, frame t): the
+// f x 128-byte tile of frame t.  Every CTA takes a contiguous run of units in (slice-major,
+// frame-minor) order, so it walks consecutive frames of one slice; several CTAs share an SM and
+// cover each other's waits.
 //
-//   score_pass_kernel      512 threads in two roles that meet at hardware barriers:
-//       row warps (up to 12; 16 lanes per row, one 16-byte vector per lane, two rows per warp
-//                          and visit) keep the frame they saw last in registers, already widened
-//                          to fp32, and the vectors of the next tile on their way in from global
-//                          memory (one 128-bit streaming load per row and lane, issued a whole
-//                          tile ahead).  A tile is visited once: each element is widened once and
-//                          feeds ||a||^2, the column sums of the tile and ||a - b||^2 against the
-//                          registers, which it then replaces.  While the helper turns the column
-//                          sums into the frame mean the warp adds up its row sums over the 16
-//                          lanes of a row (through its own patch of shared memory); then it takes
-//                          <a, mean> from the registers and writes one record of partial sums per
-//                          row and slice.
-//       helper warps (4)   add up the column sums the row warps leave in shared memory, publish
-//                          the slice of the frame mean and tell the row warps what the next unit is.
-//       No thread ever spins: the roles wait for each other at bar.sync only.
+//   score_pass_kernel   Up to 8 warps; a warp covers 4 rows per visit (8 lanes per row, one 16-byte
+//       vector per lane) and a tile in R visits.  A thread owns the same (row, vector) positions in
+//       every tile of the run:
+//         - the tile it saw last stays, as stored, in the thread's own slots of shared memory,
+//         - the tile it is about to see is on its way from global memory into registers (128-bit
+//           streaming loads issued a whole tile ahead).
+//       One visit per tile: the new vector a and the stored vector b of the frame in front are
+//       widened once and feed ||a||^2, the column sums of the tile, ||a - b||^2 and <b, mean of b's
+//       frame> (the mean term of a tile is taken one tile late, when its column sums have become the
+//       frame mean, so no warp waits for the mean inside a tile).  Row sums cross the 8 lanes of a row
+//       through the warp's own patch of shared memory.  Per row and slice three partial sums go to
+//       the workspace.  Two block barriers per tile; nothing polls.
+//       The kernel never looks at the video table: the temporal partial sum of a frame that opens a
+//       video is computed against whatever tile was in front and ignored by the finaliser.
 //   score_finalize_kernel  one CTA per frame, launched as a programmatic dependent so that its
 //       start-up overlaps the tail of the pass: adds the slices in a fixed order and writes
 //       S, T, I, the ratio and the budget of the frame.
@@ -28,15 +28,12 @@
 namespace sharpv {
 namespace {
 
-constexpr int kSliceBytes = 256;
-constexpr int kMaxRowWarps = 12;        // a row warp = 2 rows x 16 lanes (one vector per lane)
-constexpr int kHelpWarps = 4;
-constexpr int kRowThreads = kMaxRowWarps * 32;      // three warpgroups; warps beyond W stay idle
-constexpr int kHelpThreads = kHelpWarps * 32;
-constexpr int kThreads = kRowThreads + kHelpThreads;
-constexpr int kMaxVisits = 11;          // rows a half warp keeps in registers
+constexpr int kSliceBytes = 128;
+constexpr int kMaxWarps = 8;            // a warp = 4 rows x 8 lanes (one vector per lane) per visit
+constexpr int kMaxVisits = 8;           // rows a lane group walks per tile
 constexpr int kMaxTokensFused = 256;    // the finaliser takes one row per thread of a 256-thread group
-static_assert(2 * kMaxRowWarps * kMaxVisits >= kMaxTokensFused, "the row warps must cover the largest frame");
+static_assert(4 * kMaxWarps * kMaxVisits >= kMaxTokensFused, "the warps must cover the largest frame");
+constexpr int kRedStride = 9;           // floats per (visit, row) slot of a warp's patch: 8 lane parts + 1 pad
 constexpr int kFinThreads = 1024;
 
 struct FusedParams {
@@ -50,14 +47,13 @@ struct FusedParams {
     float *out_I, *out_S, *out_T, *out_ratio;
     int32_t* out_k;
     float* mean;            // [F, d]
-    float4* part;           // [F, nsl, f]: (||a||^2, <a, m>, ||a-b||^2, ||b||^2) of the slice
-    int W;                  // row warps at work: a tile is covered in R = ceil(f / 2W) visits
+    float4* part;           // [F, nsl, f]: (||a||^2, <a, mean>, ||a-b||^2, ||b||^2) of the row's part in the slice,
+                            // b = the same position one frame earlier
+    int W;                  // warps per CTA: a tile is covered in R = ceil(f / 4W) visits
 };
 
-// Hardware barriers between the roles: the side that hands something over arrives, the side that
-// needs it syncs; `threads` counts both sides.  A warp that waits here issues nothing meanwhile.
-constexpr int kBarSums = 1;     // column sums of a tile are in colp (row warps -> helper warps)
-constexpr int kBarMean = 2;     // frame mean of a tile and the next unit's tag are out (helper -> row warps)
+constexpr int kBarSums = 1;     // the column sums of a tile are in shared memory
+constexpr int kBarMean = 2;     // the frame-mean slice of a tile is in shared memory
 __device__ __forceinline__ void bar_arrive(int id, int threads) {
     asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -72,9 +68,12 @@ __device__ __forceinline__ f32x2 pk(float lo, float hi) {
     asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
     return r;
 }
+__device__ __forceinline__ void unpk(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
 __device__ __forceinline__ float hsum(f32x2 v) {
     float lo, hi;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+    unpk(v, lo, hi);
     return lo + hi;
 }
 __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
@@ -108,336 +107,273 @@ __device__ __forceinline__ f32x2 pair_f32(uint32_t lo, uint32_t hi) {
     return r;
 }
 
+template <int DT> struct Pairs;
+template <> struct Pairs<SHARPV_BF16> {
+    static constexpr int H = 4;     // fp32 pairs per 16-byte vector
+    __device__ __forceinline__ static void widen(const uint4& v, f32x2 (&o)[4]) {
+        o[0] = widen_bf16x2(v.x); o[1] = widen_bf16x2(v.y); o[2] = widen_bf16x2(v.z); o[3] = widen_bf16x2(v.w);
+    }
+};
+template <> struct Pairs<SHARPV_F32> {
+    static constexpr int H = 2;
+    __device__ __forceinline__ static void widen(const uint4& v, f32x2 (&o)[2]) {
+        o[0] = pair_f32(v.x, v.y); o[1] = pair_f32(v.z, v.w);
+    }
+};
+
+__device__ __forceinline__ f32x2 shfl_xor2(f32x2 v, int mask) {
+    float lo, hi;
+    unpk(v, lo, hi);
+    lo = __shfl_xor_sync(0xffffffffu, lo, mask);
+    hi = __shfl_xor_sync(0xffffffffu, hi, mask);
+    return pk(lo, hi);
+}
+
+
 __device__ __forceinline__ bool frame_is_first(const int32_t* vfo, int num_videos, int t) {
     const int b = upper_segment(vfo, num_videos, t);
     return __ldg(vfo + b) == t;
 }
 
-// where a CTA stands in its range of units
-struct Walk {
-    int s, t;           // slice and frame of the current unit
-    int vid, next_start;
-    bool is_first;      // frame t opens a video
-
-    __device__ __forceinline__ void start(const FusedParams& p, int64_t u0) {
-        s = (int)(u0 / p.F);
-        t = (int)(u0 % p.F);
-        vid = upper_segment(p.video_frame_offsets, p.num_videos, t);
-        is_first = __ldg(p.video_frame_offsets + vid) == t;
-        next_start = __ldg(p.video_frame_offsets + vid + 1);
-    }
-    // advances to the next unit; returns true when it starts a new slice
-    __device__ __forceinline__ bool step(const FusedParams& p) {
-        if (++t == p.F) {
-            t = 0;
-            ++s;
-            vid = upper_segment(p.video_frame_offsets, p.num_videos, 0);
-            next_start = __ldg(p.video_frame_offsets + vid + 1);
-            is_first = true;
-            return true;
-        }
-        is_first = false;
-        while (t >= next_start && vid + 1 < p.num_videos) {         // skips videos without frames
-            ++vid;
-            is_first = true;
-            next_start = __ldg(p.video_frame_offsets + vid + 1);
-        }
-        return false;
-    }
-};
-
-
-// Shared memory of one CTA (about 40 KB).
-template <int DT>
-struct Smem {
-    static constexpr int SE = kSliceBytes / Elem<DT>::kBytes;   // elements per slice row
-    static constexpr int kRedStride = 66;                       // floats per visit slot: a float2 per lane, and 2 so that the slots start on different banks
-    static constexpr int kRedFloats = 16 * kRedStride;          // per row warp: 16 visit slots
-    float colp[2 * kMaxRowWarps * SE];      // column sums of each half warp, lane-major order
-    float red[kMaxRowWarps * kRedFloats];   // row sums of each warp on their way across lanes
-    float mean_s[SE];                       // frame-mean slice of the newest tile, same order as colp
-    int2 info[2];                           // of unit n, at n & 1: t * nsl + s, "opens a video"
-};
-
-// Order of the SE floats of a slice row in colp / mean_s: float 4k + q of lane j's vector sits at
-// (16k + j) * 4 + q, so that the 16 lanes of a row store and load whole float4s side by side.
-// Returns the column of the slice that position `off` holds.
-template <int DT>
-__device__ __forceinline__ int column_of_position(int off) {
-    constexpr int P = Elem<DT>::kPerVec;
-    const int q = off & 3, j = (off >> 2) & 15, k = off >> 6;
-    return j * P + 4 * k + q;
-}
-
-template <int DT>
-__device__ __forceinline__ void widen_pairs(const uint4& v, f32x2 (&o)[Elem<DT>::kPerVec / 2]) {
-    constexpr int H = Elem<DT>::kPerVec / 2;
-    if (DT == SHARPV_BF16) {
-        o[0] = widen_bf16x2(v.x); o[1] = widen_bf16x2(v.y);
-        o[H - 2] = widen_bf16x2(v.z); o[H - 1] = widen_bf16x2(v.w);
-    } else {
-        o[0] = pair_f32(v.x, v.y); o[H - 1] = pair_f32(v.z, v.w);
-    }
-}
-
-// ---------------------------------------------------------------------------------------
-// helper warps: frame mean, unit tags
-// ---------------------------------------------------------------------------------------
-template <int DT>
-__device__ __forceinline__ void helper_role(const FusedParams& p, Smem<DT>& sm, int64_t u0, int n_units, int htid) {
-    constexpr int SE = Smem<DT>::SE;
-    Walk w;
-    w.start(p, u0);
-    const int column = column_of_position<DT>(htid & (SE - 1));
-    float* mean_out = p.mean + (int64_t)w.t * p.d + w.s * SE + column;
-    const float* my_col = sm.colp + htid;
-    const int groups = 2 * p.W;
-    const int both = 32 * p.W + kHelpThreads;
-    const float ff = (float)p.f;
-    if (htid == 0) sm.info[0] = make_int2(w.t * p.nsl + w.s, w.is_first ? 1 : 0);
-    bar_arrive(kBarMean, both);                 // the first unit's tag is out
-    for (int n = 0; n < n_units; ++n) {
-        float* out = mean_out;
-        if (w.step(p)) mean_out = p.mean + w.s * SE + column;
-        else mean_out += p.d;
-        if (htid == 0) sm.info[(n + 1) & 1] = make_int2(w.t * p.nsl + w.s, w.is_first ? 1 : 0);
-        bar_sync(kBarSums, both);
-        if (htid < SE) {
-            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-            int gidx = 0;
-#pragma unroll 2
-            for (; gidx + 3 < groups; gidx += 4) {
-                s0 += my_col[(gidx + 0) * SE];
-                s1 += my_col[(gidx + 1) * SE];
-                s2 += my_col[(gidx + 2) * SE];
-                s3 += my_col[(gidx + 3) * SE];
-            }
-            if (gidx < groups) {            // groups is even
-                s0 += my_col[(gidx + 0) * SE];
-                s1 += my_col[(gidx + 1) * SE];
-            }
-            const float m = ((s0 + s1) + (s2 + s3)) / ff;
-            sm.mean_s[htid] = m;
-            *out = m;
-        }
-        bar_arrive(kBarMean, both);
-    }
-}
-
-// ---------------------------------------------------------------------------------------
-// row warps
-// ---------------------------------------------------------------------------------------
-// Lane (g, j) of warp `warp` (g = lane / 16) owns, in visit v, vector j of row 2 W v + 2 warp + g.
-// Visits below R - 1 exist for every warp and every lane; in the last one a warp takes part if its
-// first row exists, and a half warp whose own row lies beyond the frame loads nothing and works on
-// zeros.
-//
-// Row sums cross the 16 lanes of a row through the warp's own patch of shared memory: every lane
-// leaves its parts there, then lane l adds up the 16 parts of row l / 16, visit l % 16 of the warp,
-// in lane order.
-template <int DT, int R>
-struct RowRegs {
-    static constexpr int H = Elem<DT>::kPerVec / 2;
-    static constexpr int kRS = 66;      // floats per visit slot of the warp's patch (Smem::kRedStride)
-    f32x2 prev[R][H];       // the frame seen last, fp32 pairs: [visit][pair]
-    uint4 raw[R];           // the tile about to be visited, as it arrives from global memory
-
-    __device__ __forceinline__ void clear() {
-#pragma unroll
-        for (int v = 0; v < R; ++v) {
-            raw[v] = make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-            for (int i = 0; i < H; ++i) prev[v][i] = pk(0.f, 0.f);
-        }
-    }
-
-    // requests this lane's vectors of the tile at `tile` (this lane's first row and column)
-    __device__ __forceinline__ void request(const char* tile, int64_t vstride, bool last_mine) {
-#pragma unroll
-        for (int v = 0; v < R; ++v)
-            if (v < R - 1 || last_mine) raw[v] = __ldcs(reinterpret_cast<const uint4*>(tile + v * vstride));
-    }
-
-    // One visit of the tile in `raw`: ||a||^2 and ||a - b||^2 (TEMPORAL, b = the rows in registers)
-    // of this lane's part of each row go to the warp's patch, col += a (COLS), the registers then
-    // hold the new rows, and the vectors of the tile behind it (`next`, if any) are requested as
-    // soon as a register is free for them.
-    template <bool TEMPORAL, bool COLS>
-    __device__ __forceinline__ void take_tile(const char* next, int64_t vstride, bool last_warp, bool last_mine,
-                                              f32x2 (&col)[H], float* red_lane) {
-#pragma unroll
-        for (int v = 0; v < R; ++v) {
-            if (v < R - 1 || last_warp) {
-                f32x2 a2[H];
-                widen_pairs<DT>(raw[v], a2);
-                if (next && (v < R - 1 || last_mine)) raw[v] = __ldcs(reinterpret_cast<const uint4*>(next));
-                next += vstride;
-                f32x2 aa, db;
-#pragma unroll
-                for (int i = 0; i < H; ++i) {
-                    aa = i == 0 ? mul2(a2[i], a2[i]) : fma2(a2[i], a2[i], aa);
-                    if (COLS) col[i] = (v == 0 && R > 1) ? a2[i] : add2(col[i], a2[i]);
-                    if (TEMPORAL) {
-                        const f32x2 e = sub2(a2[i], prev[v][i]);
-                        db = i == 0 ? mul2(e, e) : fma2(e, e, db);
-                    }
-                    prev[v][i] = a2[i];
-                }
-                *reinterpret_cast<float2*>(red_lane + v * kRS) = make_float2(hsum(aa), TEMPORAL ? hsum(db) : 0.f);
-            }
-        }
-    }
-
-    // <a, mean> of the rows in registers, this lane's part of each row, to the warp's patch
-    __device__ __forceinline__ void against_mean(const f32x2 (&m)[H], bool last_warp, int g, float* red_lane) const {
-#pragma unroll
-        for (int v = 0; v < R; ++v) {
-            if (v < R - 1 || last_warp) {
-                f32x2 am;
-#pragma unroll
-                for (int i = 0; i < H; ++i) am = i == 0 ? mul2(prev[v][i], m[i]) : fma2(prev[v][i], m[i], am);
-                red_lane[v * kRS + g] = hsum(am);
-            }
-        }
-    }
-};
-
-template <int DT, int R>
-__device__ __forceinline__ void row_role(const FusedParams& p, Smem<DT>& sm, int64_t u0, int n_units, int halo,
-                                         int tid) {
-    constexpr int H = Elem<DT>::kPerVec / 2, SE = Smem<DT>::SE;
-    static_assert(H >= 2, "two accumulators per sum");
-    const int lane = tid & 31, warp = tid >> 5, g = lane >> 4, j = lane & 15;
-    const int row0 = 2 * warp + g;
-    const bool last_warp = 2 * p.W * (R - 1) + 2 * warp < p.f;      // the warp takes part in the last visit
-    const bool last_mine = 2 * p.W * (R - 1) + row0 < p.f;          // and this lane's own row exists there
-    const int64_t vstride = (int64_t)2 * p.W * p.row_bytes_ld;
-    const int64_t frame_bytes = (int64_t)p.f * p.row_bytes_ld;
-    float* my_colp = sm.colp + (2 * warp + g) * SE + j * 4;         // float4 k of this lane at + 64 k
-    const float* my_mean = sm.mean_s + j * 4;
-    float* red_warp = sm.red + warp * Smem<DT>::kRedFloats;
-    float* red_lane = red_warp + lane * 2;                          // visit v of this lane at + 64 v
-    // the row sums this lane adds up: row sg of the warp's two, visit sv, starting with lane srot
-    const int sg = lane >> 4, sv = lane & 15;
-    const float* sum_src = red_warp + sv * Smem<DT>::kRedStride + sg * 32;    // float2 of lane j' of the row at + 2 j'
-    const int my_row = 2 * p.W * sv + 2 * warp + sg;
-    const bool sums = sv < R;
-    const bool writes = sums && my_row < p.f;
-    const int both = 32 * p.W + kHelpThreads;
-
-    RowRegs<DT, R> st;
-    st.clear();
-    float prev_aa = 0.f;            // ||row||^2 of the frame seen last, for the row this lane adds up
-
-    // this lane's first vector of the first tile: the frame in front of the range, if it matters
-    const int s0 = (int)(u0 / p.F);
-    int t = (int)(u0 % p.F) - halo;
-    const char* tile = p.tokens + ((int64_t)t * p.f + row0) * p.row_bytes_ld + (int64_t)s0 * kSliceBytes + j * 16;
-    st.request(tile, vstride, last_mine);
-    bar_sync(kBarMean, both);                   // the first unit's tag
-    const int Q = n_units + halo;
-    int n = 0;
-    for (int q = 0; q < Q; ++q) {
-        const bool halo_tile = halo && q == 0;
-        // the tile behind this one: the next frame of the slice, or the first frame of the next slice
-        const char* next = nullptr;
-        if (q + 1 < Q) {
-            if (++t == p.F) {
-                t = 0;
-                next = tile - (int64_t)(p.F - 1) * frame_bytes + kSliceBytes;
-            } else {
-                next = tile + frame_bytes;
-            }
-        }
-        const int2 inf = sm.info[n & 1];
-        const bool temporal = !halo_tile && inf.y == 0;     // the frame continues a video
-        f32x2 col[H];
-        if (R == 1) {               // the only visit may be one this warp has no part in
-#pragma unroll
-            for (int i = 0; i < H; ++i) col[i] = pk(0.f, 0.f);
-        }
-        if (halo_tile) st.template take_tile<false, false>(next, vstride, last_warp, last_mine, col, red_lane);
-        else if (temporal) st.template take_tile<true, true>(next, vstride, last_warp, last_mine, col, red_lane);
-        else st.template take_tile<false, true>(next, vstride, last_warp, last_mine, col, red_lane);
-        tile = next;
-        if (!halo_tile) {
-#pragma unroll
-            for (int k = 0; k < H / 2; ++k)
-                *reinterpret_cast<ulonglong2*>(my_colp + 64 * k) = make_ulonglong2(col[2 * k], col[2 * k + 1]);
-            bar_arrive(kBarSums, both);                     // the column sums are out
-        }
-        __syncwarp();
-        // row sums of ||a||^2 and ||a - b||^2 while the helper makes the mean
-        f32x2 xy = pk(0.f, 0.f);
-        if (sums) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i)
-                xy = add2(xy, *reinterpret_cast<const f32x2*>(sum_src + 2 * i));
-        }
-        __syncwarp();                                       // the patch is free again
-        float my_aa, my_db;
-        asm("mov.b64 {%0, %1}, %2;" : "=f"(my_aa), "=f"(my_db) : "l"(xy));
-
-        if (!halo_tile) {
-            bar_sync(kBarMean, both);
-            f32x2 m[H];
-#pragma unroll
-            for (int k = 0; k < H / 2; ++k) {
-                const ulonglong2 x = *reinterpret_cast<const ulonglong2*>(my_mean + 64 * k);
-                m[2 * k] = x.x;
-                m[2 * k + 1] = x.y;
-            }
-            st.against_mean(m, last_warp, g, red_lane);
-            __syncwarp();
-            float my_am = 0.f;
-            if (sums) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) my_am += sum_src[2 * i + sg];
-            }
-            __syncwarp();                                   // the patch is free again
-            if (writes)
-                p.part[(int64_t)inf.x * p.f + my_row] = make_float4(my_aa, my_am, my_db, temporal ? prev_aa : 0.f);
-            ++n;
-        }
-        prev_aa = my_aa;
-    }
+// Shared memory of one CTA of W warps and R visits, in this order:
+//   float2 red2[W][4 R * 9]       per warp: lane parts of (||a||^2, ||a-b||^2)
+//   float  red1[W][4 R * 9]       per warp: lane parts of <b, mean>
+//   float  colp[W][SE]            per warp: column sums of the tile
+//   float  mean_s[SE]             frame-mean slice of the newest tile
+constexpr size_t pass_smem_bytes(int W, int R, int SE) {
+    return (size_t)W * 4 * R * kRedStride * 12 + (size_t)W * SE * 4 + (size_t)SE * 4;
 }
 
 template <int DT, int R>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(32 * kMaxWarps, 2)
 score_pass_kernel(const FusedParams p) {
+    constexpr int H = Pairs<DT>::H;
+    constexpr int P = Elem<DT>::kPerVec;
+    constexpr int SE = kSliceBytes / Elem<DT>::kBytes;      // elements per slice row
+    constexpr int kPlane = 4 * R * kRedStride;              // slots of a warp's patch
+    constexpr int D = R >= 6 ? 1 : 0;                     // visits by which the hand-over of a register lags
     extern __shared__ __align__(16) unsigned char smem[];
-    Smem<DT>& sm = *reinterpret_cast<Smem<DT>*>(smem);
+
+    const int W = p.W, NT = 32 * W;
+    float2* red2 = reinterpret_cast<float2*>(smem);
+    float* red1 = reinterpret_cast<float*>(red2 + W * kPlane);
+    float* colp = red1 + W * kPlane;
+    float* mean_s = colp + W * SE;
 
     cudaGridDependencySynchronize();        // the tokens come from earlier work on the stream
     // Let the finaliser's CTAs be scheduled as soon as SMs free up; they wait for this whole grid.
-    // Only after the wait above: what the finaliser reads before its own wait (the frame table) is
-    // then known to be complete.
     cudaTriggerProgrammaticLaunchCompletion();
     const int64_t U = (int64_t)p.nsl * p.F;
     const int64_t u0 = U * blockIdx.x / gridDim.x;
     const int64_t u1 = U * (blockIdx.x + 1) / gridDim.x;
     if (u0 >= u1) return;
     const int n_units = (int)(u1 - u0);
-    const int t0 = (int)(u0 % p.F);
-    const int vid0 = upper_segment(p.video_frame_offsets, p.num_videos, t0);
-    const int halo = (__ldg(p.video_frame_offsets + vid0) == t0) ? 0 : 1;
+    int s = (int)(u0 / p.F), t = (int)(u0 % p.F);
 
-    // The block is launched with 128 registers per thread (512 x 128 = 65536).  The helper warps give
-    // most of theirs back and the three row warpgroups take them: 128 x 32 + 384 x 160 = 65536.
-    const int tid = threadIdx.x;
-    if (tid < kRowThreads) {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 160;");
-        if ((tid >> 5) < p.W) row_role<DT, R>(p, sm, u0, n_units, halo, tid);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 3, j = lane & 7;
+    const int row0 = 4 * warp + g;                                  // this lane's row in visit 0
+    const bool last_mine = (R - 1) * 4 * W + row0 < p.f;            // its row of the last visit exists
+    const bool last_warp = (R - 1) * 4 * W + 4 * warp < p.f;        // the warp has a row in the last visit
+    const int64_t vstride = (int64_t)4 * W * p.row_bytes_ld;
+    const int64_t frame_bytes = (int64_t)p.f * p.row_bytes_ld;
+    float2* red2_lane = red2 + warp * kPlane + g * kRedStride + j;  // visit v at + 4 v * kRedStride
+    float* red1_lane = red1 + warp * kPlane + g * kRedStride + j;
+    // the row sums this lane adds up: visit sv, row sg of the warp's four
+    const int sv = lane >> 2, sg = lane & 3;
+    const float2* sum2_src = red2 + warp * kPlane + lane * kRedStride;
+    const float* sum1_src = red1 + warp * kPlane + lane * kRedStride;
+    const int my_row = sv * 4 * W + 4 * warp + sg;
+    const bool sums = sv < R;
+    const bool writes = sums && my_row < p.f;
+    const int mean_warps = W < SE / 32 ? W : SE / 32;               // warps that turn column sums into the mean
+    const float inv_f = 1.f / (float)p.f;
+
+    // Two tiles live in registers as stored: the one being visited and the one in front of it.  The
+    // registers of the one in front are handed, vector by vector, to the tile behind, so the names
+    // swap from tile to tile and nothing is copied.
+    uint4 ta[R], tb[R];
+    const char* nxt = p.tokens + ((int64_t)t * p.f + row0) * p.row_bytes_ld + (int64_t)s * kSliceBytes + j * 16;
+#pragma unroll
+    for (int v = 0; v < R; ++v) {
+        const bool mine = v < R - 1 || last_mine;
+        ta[v] = make_uint4(0u, 0u, 0u, 0u);
+        tb[v] = make_uint4(0u, 0u, 0u, 0u);
+        if (mine) ta[v] = __ldcs(reinterpret_cast<const uint4*>(nxt + v * vstride));
+        if (mine && t > 0) tb[v] = __ldcs(reinterpret_cast<const uint4*>(nxt - frame_bytes + v * vstride));
+    }
+
+    f32x2 m[H];                     // this lane's columns of the mean of the frame in front
+#pragma unroll
+    for (int i = 0; i < H; ++i) m[i] = pk(0.f, 0.f);
+    int t_prev = t, s_prev = s;
+
+    // What the lane that adds up a row keeps from tile to tile: ||a||^2 and ||a-b||^2 of the tile seen
+    // last (its record is written one tile late, together with its mean term) and that tile's ||b||^2,
+    // which is the ||a||^2 of the tile before it.  For the first tile of the run that is the frame in
+    // front of the run, still in `tb`.
+    float keep_aa = 0.f, keep_db = 0.f, keep_bb = 0.f;
+    if (t > 0) {
+#pragma unroll
+        for (int v = 0; v < R; ++v) {
+            f32x2 b2[H];
+            Pairs<DT>::widen(tb[v], b2);
+            f32x2 bb;
+#pragma unroll
+            for (int i = 0; i < H; ++i) bb = i == 0 ? mul2(b2[i], b2[i]) : fma2(b2[i], b2[i], bb);
+            red1_lane[4 * v * kRedStride] = hsum(bb);
+        }
+        __syncwarp();
+        if (sums) {
+            float x = sum1_src[0];
+#pragma unroll
+            for (int i = 1; i < 8; ++i) x += sum1_src[i];
+            keep_aa = x;
+        }
+        __syncwarp();
+    }
+
+    // One tile: `cur` is visited against `old`; the registers of `old` receive the tile behind `cur`.
+    auto visit_tile = [&](uint4 (&cur)[R], uint4 (&old)[R], int n) {
+        // the tile behind this one: the next frame of the slice, or the first frame of the next slice
+        const bool has_next = n + 1 < n_units;
+        int t_next = t + 1, s_next = s;
+        if (t_next == p.F) {
+            t_next = 0;
+            s_next = s + 1;
+            nxt += kSliceBytes - (int64_t)(p.F - 1) * frame_bytes;
+        } else {
+            nxt += frame_bytes;
+        }
+        const char* q = nxt;
+
+        f32x2 col[H];
+#pragma unroll
+        for (int v = 0; v < R; ++v) {
+            const bool active = v < R - 1 || R == 1 || last_warp;   // warp-uniform
+            f32x2 a2[H], b2[H];
+            if (active) {
+                Pairs<DT>::widen(cur[v], a2);
+                Pairs<DT>::widen(old[v], b2);
+            }
+            if (v >= D) {
+                if (has_next && (v - D < R - 1 || last_mine)) old[v - D] = __ldcs(reinterpret_cast<const uint4*>(q));
+                q += vstride;
+            }
+            if (active) {
+                f32x2 aa, db, bm;
+#pragma unroll
+                for (int i = 0; i < H; ++i) {
+                    aa = i == 0 ? mul2(a2[i], a2[i]) : fma2(a2[i], a2[i], aa);
+                    col[i] = v == 0 ? a2[i] : add2(col[i], a2[i]);
+                    const f32x2 e = sub2(a2[i], b2[i]);
+                    db = i == 0 ? mul2(e, e) : fma2(e, e, db);
+                    bm = i == 0 ? mul2(b2[i], m[i]) : fma2(b2[i], m[i], bm);
+                }
+                red2_lane[4 * v * kRedStride] = make_float2(hsum(aa), hsum(db));
+                red1_lane[4 * v * kRedStride] = hsum(bm);
+            }
+        }
+#pragma unroll
+        for (int v = R - D; v < R; ++v) {
+            if (v >= 0) {
+                if (has_next && (v < R - 1 || last_mine)) old[v] = __ldcs(reinterpret_cast<const uint4*>(q));
+                q += vstride;
+            }
+        }
+        // column sums of the warp's four row groups, then one partial per warp
+#pragma unroll
+        for (int i = 0; i < H; ++i) {
+            col[i] = add2(col[i], shfl_xor2(col[i], 8));
+            col[i] = add2(col[i], shfl_xor2(col[i], 16));
+        }
+        if (lane < 8) {
+            float* dst = colp + warp * SE + lane * P;
+#pragma unroll
+            for (int i = 0; i < H; i += 2)
+                *reinterpret_cast<ulonglong2*>(dst + 2 * i) = make_ulonglong2(col[i], col[i + 1]);
+        }
+        if (warp >= mean_warps) bar_arrive(kBarSums, NT);
+        __syncwarp();
+        // row sums over the 8 lanes of a row
+        if (sums) {
+            f32x2 x2 = *reinterpret_cast<const f32x2*>(sum2_src);
+            float xm = sum1_src[0];
+#pragma unroll
+            for (int i = 1; i < 8; ++i) {
+                x2 = add2(x2, *reinterpret_cast<const f32x2*>(sum2_src + i));
+                xm += sum1_src[i];
+            }
+            float xa, xd;
+            unpk(x2, xa, xd);
+            if (writes && n > 0)
+                p.part[((int64_t)t_prev * p.nsl + s_prev) * p.f + my_row] = make_float4(keep_aa, xm, keep_db, keep_bb);
+            keep_bb = keep_aa;
+            keep_aa = xa;
+            keep_db = xd;
+        }
+        if (warp < mean_warps) {
+            bar_sync(kBarSums, NT);
+            float* mean_out = p.mean + (int64_t)t * p.d + s * SE;
+            for (int c = tid; c < SE; c += 32 * mean_warps) {
+                float acc = colp[c];
+                for (int q2 = 1; q2 < W; ++q2) acc += colp[q2 * SE + c];
+                acc *= inv_f;
+                mean_s[c] = acc;
+                mean_out[c] = acc;
+            }
+        }
+        bar_sync(kBarMean, NT);
+        {
+            const float* src = mean_s + j * P;
+#pragma unroll
+            for (int i = 0; i < H; i += 2) {
+                const ulonglong2 x = *reinterpret_cast<const ulonglong2*>(src + 2 * i);
+                m[i] = x.x;
+                m[i + 1] = x.y;
+            }
+        }
+        t_prev = t;
+        s_prev = s;
+        t = t_next;
+        s = s_next;
+    };
+
+    // the mean term of the last tile of the run
+    auto last_mean_term = [&](const uint4 (&last)[R]) {
+#pragma unroll
+        for (int v = 0; v < R; ++v) {
+            f32x2 b2[H];
+            Pairs<DT>::widen(last[v], b2);
+            f32x2 bm;
+#pragma unroll
+            for (int i = 0; i < H; ++i) bm = i == 0 ? mul2(b2[i], m[i]) : fma2(b2[i], m[i], bm);
+            red1_lane[4 * v * kRedStride] = hsum(bm);
+        }
+        __syncwarp();
+        if (writes) {
+            float xm = sum1_src[0];
+#pragma unroll
+            for (int i = 1; i < 8; ++i) xm += sum1_src[i];
+            p.part[((int64_t)t_prev * p.nsl + s_prev) * p.f + my_row] = make_float4(keep_aa, xm, keep_db, keep_bb);
+        }
+    };
+
+    int n = 0;
+    for (; n + 1 < n_units; n += 2) {
+        visit_tile(ta, tb, n);
+        visit_tile(tb, ta, n + 1);
+    }
+    if (n < n_units) {
+        visit_tile(ta, tb, n);
+        last_mean_term(ta);
     } else {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 32;");
-        helper_role<DT>(p, sm, u0, n_units, tid - kRowThreads);
+        last_mean_term(tb);
     }
 }
 
 // One CTA per frame: adds the slices in a fixed order, writes S, T, I, ratio_t and k_t.
-// 1024 threads = 4 groups x 256 rows; group q adds slices q, q+4, ... (all loads in flight at once),
-// then the four group sums are added in order.
+// 1024 threads = 4 groups x 256 rows; group q adds slices q, q+4, ... (up to 8 records in flight per
+// thread), then the four group sums are added in order.
 template <int DT>
 __global__ void __launch_bounds__(kFinThreads)
 score_finalize_kernel(const FusedParams p) {
@@ -452,9 +388,8 @@ score_finalize_kernel(const FusedParams p) {
     // everything the pass kernel wrote is visible after this point
     cudaGridDependencySynchronize();
 
-    // every load of this thread is issued before the first one is used: one memory round trip
     const float* mean = p.mean + (int64_t)t * p.d;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);       // ||a||^2, <a, mean>, ||a - b||^2, ||b||^2
     float sm = 0.f;
     const float4* src = p.part + ((int64_t)t * p.nsl) * p.f + row;
     for (int s0 = grp; s0 < p.nsl; s0 += 32) {
@@ -466,8 +401,8 @@ score_finalize_kernel(const FusedParams p) {
         }
         if (s0 == grp) {
             for (int c = tid * 4; c < p.d; c += kFinThreads * 4) {
-                const float4 m = __ldcg(reinterpret_cast<const float4*>(mean + c));
-                sm = fmaf(m.x, m.x, sm); sm = fmaf(m.y, m.y, sm); sm = fmaf(m.z, m.z, sm); sm = fmaf(m.w, m.w, sm);
+                const float4 mm = __ldcg(reinterpret_cast<const float4*>(mean + c));
+                sm = fmaf(mm.x, mm.x, sm); sm = fmaf(mm.y, mm.y, sm); sm = fmaf(mm.z, mm.z, sm); sm = fmaf(mm.w, mm.w, sm);
             }
         }
 #pragma unroll
@@ -486,7 +421,7 @@ score_finalize_kernel(const FusedParams p) {
         const float aa = (a0.x + a1.x) + (a2.x + a3.x), am = (a0.y + a1.y) + (a2.y + a3.y);
         const float db = (a0.z + a1.z) + (a2.z + a3.z), bb = (a0.w + a1.w) + (a2.w + a3.w);
         const float s2 = dissim_sq_from_dot(aa, smm, am);
-        const float t2 = is_first ? 0.f : dissim_sq_from_sums(aa, bb, db);
+        const float t2 = is_first ? 0.f : dissim_sq_from_sums(aa, bb, db);      // a video's first frame: db, bb unused
         int fl = 0;
         if (s2 < kRefineBelowDot) fl |= 1;
         if (!is_first && t2 < kRefineBelow && db != 0.f) fl |= 2;
@@ -534,41 +469,46 @@ score_finalize_kernel(const FusedParams p) {
     }
 }
 
-// The split of a frame over the row warps: W warps cover 2W rows a visit and the frame in
-// R = ceil(f / 2W) visits; warp w sits on scheduler w mod 4.  The split with the lightest
-// busiest scheduler wins, then the larger W.
+// The split of a frame over the warps of a CTA: W warps of 4 rows a visit, R = ceil(f / 4W) visits.
+// The split with the fewest warp-visits wins (no warp idles through a visit), then the one with
+// fewer visits.
 void row_split(int f, int& W, int& R) {
     int best = 1 << 30;
-    W = kMaxRowWarps;
+    W = kMaxWarps;
     R = kMaxVisits;
-    for (int w = 1; w <= kMaxRowWarps; ++w) {
-        const int r = (f + 2 * w - 1) / (2 * w);
+    for (int w = 1; w <= kMaxWarps; ++w) {
+        const int r = (f + 4 * w - 1) / (4 * w);
         if (r > kMaxVisits) continue;
-        int load[4] = {0, 0, 0, 0};
-        for (int i = 0; i < w; ++i) load[i & 3] += r - 1 + (2 * w * (r - 1) + 2 * i < f ? 1 : 0);
-        int worst = 0;
-        for (int k = 0; k < 4; ++k) worst = load[k] > worst ? load[k] : worst;
-        if (worst <= best) { best = worst; W = w; R = r; }
+        if (w * r < best || (w * r == best && r < R)) { best = w * r; W = w; R = r; }
     }
 }
 
 template <int DT, int R>
-sharpv_status launch(const FusedScoreArgs& a, FusedParams& p, int sms) {
-    const size_t smem = sizeof(Smem<DT>);
-    if (cudaFuncSetAttribute(score_pass_kernel<DT, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess) {
-        (void)cudaGetLastError();
-        return SHARPV_ERR_UNSUPPORTED;
+sharpv_status launch(const FusedScoreArgs& a, FusedParams& p, int dev, int sms) {
+    constexpr int SE = kSliceBytes / Elem<DT>::kBytes;
+    auto kernel = score_pass_kernel<DT, R>;
+    const size_t smem = pass_smem_bytes(p.W, R, SE);
+    // resident CTAs per SM of this instance and block size, asked once per device
+    static int resident[64][kMaxWarps + 1] = {};
+    if (dev < 0 || dev >= 64) return SHARPV_ERR_UNSUPPORTED;
+    int per_sm = resident[dev][p.W];
+    if (per_sm == 0) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)pass_smem_bytes(kMaxWarps, R, SE)) != cudaSuccess ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 32 * p.W, smem) != cudaSuccess ||
+            per_sm < 1) {
+            (void)cudaGetLastError();
+            return SHARPV_ERR_UNSUPPORTED;
+        }
+        resident[dev][p.W] = per_sm;
     }
     const int64_t units = (int64_t)p.nsl * a.F;
-    const unsigned grid = (unsigned)(units < sms ? units : sms);
-    if (launch_dependent(score_pass_kernel<DT, R>, dim3(grid), dim3(kThreads), smem, a.stream, p) != cudaSuccess) {
+    const int64_t slots = (int64_t)sms * per_sm;
+    const unsigned grid = (unsigned)(units < slots ? units : slots);
+    if (launch_dependent(kernel, dim3(grid), dim3(32 * p.W), smem, a.stream, p) != cudaSuccess) {
         (void)cudaGetLastError();
         return SHARPV_ERR_CUDA;
     }
-#ifdef NOFIN
-    return SHARPV_OK;
-#endif
     // the finaliser starts while the pass drains and waits for it with cudaGridDependencySynchronize
     if (launch_dependent(score_finalize_kernel<DT>, dim3((unsigned)a.F), dim3(kFinThreads), 0, a.stream, p) !=
         cudaSuccess) {
@@ -579,19 +519,16 @@ sharpv_status launch(const FusedScoreArgs& a, FusedParams& p, int sms) {
 }
 
 template <int DT>
-sharpv_status launch_visits(const FusedScoreArgs& a, FusedParams& p, int sms, int R) {
+sharpv_status launch_visits(const FusedScoreArgs& a, FusedParams& p, int dev, int sms, int R) {
     switch (R) {
-        case 1: return launch<DT, 1>(a, p, sms);
-        case 2: return launch<DT, 2>(a, p, sms);
-        case 3: return launch<DT, 3>(a, p, sms);
-        case 4: return launch<DT, 4>(a, p, sms);
-        case 5: return launch<DT, 5>(a, p, sms);
-        case 6: return launch<DT, 6>(a, p, sms);
-        case 7: return launch<DT, 7>(a, p, sms);
-        case 8: return launch<DT, 8>(a, p, sms);
-        case 9: return launch<DT, 9>(a, p, sms);
-        case 10: return launch<DT, 10>(a, p, sms);
-        case 11: return launch<DT, 11>(a, p, sms);
+        case 1: return launch<DT, 1>(a, p, dev, sms);
+        case 2: return launch<DT, 2>(a, p, dev, sms);
+        case 3: return launch<DT, 3>(a, p, dev, sms);
+        case 4: return launch<DT, 4>(a, p, dev, sms);
+        case 5: return launch<DT, 5>(a, p, dev, sms);
+        case 6: return launch<DT, 6>(a, p, dev, sms);
+        case 7: return launch<DT, 7>(a, p, dev, sms);
+        case 8: return launch<DT, 8>(a, p, dev, sms);
     }
     return SHARPV_ERR_UNSUPPORTED;
 }
@@ -630,8 +567,8 @@ sharpv_status fused_score_launch(const FusedScoreArgs& a) {
         return SHARPV_ERR_CUDA;
     int R = 0;
     row_split(a.f, p.W, R);
-    return a.dtype == SHARPV_F32 ? launch_visits<SHARPV_F32>(a, p, sms, R)
-                                 : launch_visits<SHARPV_BF16>(a, p, sms, R);
+    return a.dtype == SHARPV_F32 ? launch_visits<SHARPV_F32>(a, p, dev, sms, R)
+                                 : launch_visits<SHARPV_BF16>(a, p, dev, sms, R);
 }
 
 }  // namespace sharpv

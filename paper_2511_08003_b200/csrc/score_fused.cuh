@@ -21,8 +21,8 @@ struct FusedScoreArgs {
     cudaStream_t stream;
 };
 
-// Shapes the fused kernel covers: rows that split into 256-byte column slices and frames of at
-// most 256 tokens.  Everything else takes the three-kernel path.
+// Shapes the fused kernel covers: rows that split into 128-byte column slices and frames of at most
+// 256 tokens.  Everything else takes the three-kernel path.
 bool fused_score_supported(sharpv_dtype dtype, int f, int d);
 
 // Upper bound over both storage types.

@@ -238,6 +238,7 @@ sharpv_status select_impl(int mode, const float* importance, const int32_t* k, f
     if (mode == 1 && F > 0) {
         int32_t* counts = (int32_t*)workspace;
         count_above_kernel<<<F, kSelectThreads, 0, stream>>>(importance, K, f, counts);
+        if (launch_status() != SHARPV_OK) return SHARPV_ERR_CUDA;
         budgets = counts;
     }
     if (F == 0) {

@@ -255,6 +255,39 @@ def test_kv_compact_layouts_and_layer_range():
     np.testing.assert_array_equal(to_host(dst_tm)[:, :, :kept.size], wl.kv[:, :, :, kept].transpose(0, 1, 3, 2, 4))
 
 
+def test_kv_compact_rejects_partial_overlap_accepts_neighbours():
+    """Source and destination carved out of one allocation: caches that touch without sharing a byte are
+    compacted, a destination that starts inside the source is refused before anything is launched."""
+    wl, dw = _case("small_ragged")
+    T = wl.total_seq_tokens
+    L, _, H, _, Dh = wl.kv_shape()
+    both = torch.zeros((2 * L, 2, H, T, Dh), dtype=dw.kv.dtype, device="cuda")
+    both[:L] = dw.kv
+    src, dst = both[:L], both[L:]                          # neighbours: dst starts where src ends
+    kept = np.arange(1, T, 3, dtype=np.int32)
+    kept_d = torch.from_numpy(kept).cuda()
+    kso = torch.tensor([0, kept.size], dtype=torch.int32, device="cuda")
+    sv.sharpv_kv_compact(src, dst, kept_d, kso, capacity=T)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(to_host(dst)[:, :, :, :kept.size], wl.kv[:, :, :, kept])
+    np.testing.assert_array_equal(to_host(src), wl.kv)      # the source is untouched
+    before = to_host(both).copy()
+    shifted = both.view(-1)[Dh:Dh + src.numel()].view(src.shape)      # one row further on: shares bytes with src
+    for bad in (shifted, both[1:L + 1]):
+        with pytest.raises(sv.SharpVError) as e:
+            sv.sharpv_kv_compact(src, bad, kept_d, kso, capacity=T)
+        assert e.value.status == sv.Status.ERR_INVALID_ARG
+    with pytest.raises(sv.SharpVError):
+        ws = torch.empty(sv.sharpv_kv_compact_rope_workspace_bytes(T, Dh), dtype=torch.uint8, device="cuda")
+        sv.sharpv_kv_compact_rope(src, shifted, kept_d, kso, torch.tensor([0, T], dtype=torch.int32, device="cuda"),
+                                  T, Dh, 1.0e4, workspace=ws)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(to_host(both), before)    # nothing ran
+    # a single layer of one cache into another layer of the same allocation is fine
+    sv.sharpv_kv_compact(both, both, kept_d, kso, capacity=T, layer_begin=0, layer_end=1)     # in place
+    torch.cuda.synchronize()
+
+
 @pytest.mark.parametrize("name", ["tiny", "small_ragged", "odd_shapes", "onevision_7b"])
 @pytest.mark.parametrize("M", [0.2, 0.788])
 def test_kv_compact_in_place(name, M):

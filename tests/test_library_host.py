@@ -128,7 +128,9 @@ def test_kv_compact_rejects_bad_arguments(L):
         base.update(kw)
         return sv.KVLayout(**base)
 
-    def call(src=P, sl=None, dst=2 * P, dl=None, lb=0, le=28, kp=P, kso=P, B=1, cap=1000):
+    FAR = P + (1 << 40)         # far beyond the end of the fake source cache
+
+    def call(src=P, sl=None, dst=FAR, dl=None, lb=0, le=28, kp=P, kso=P, B=1, cap=1000):
         sl = layout() if sl is None else sl
         dl = layout() if dl is None else dl
         return L.sharpv_kv_compact(src, C.byref(sl), dst, C.byref(dl), lb, le, kp, kso, B, cap, None, None)
@@ -151,6 +153,12 @@ def test_kv_compact_rejects_bad_arguments(L):
     assert call(lb=5, le=5) == S.OK                               # empty layer range: nothing to do
     assert call(cap=0, kp=None) == S.OK
     assert L.sharpv_kv_compact(P, None, 2 * P, None, 0, 1, P, P, 1, 10, None, None) == S.ERR_INVALID_ARG
+    # a destination that shares bytes with the source without being the source: rejected, nothing launched
+    plane = 1000 * 128 * 2                                        # bytes of one (layer, K|V, head) plane
+    assert call(dst=P + 256) == S.ERR_INVALID_ARG                 # shifted by one row
+    assert call(dst=P + 3 * plane) == S.ERR_INVALID_ARG           # starts inside the source cache
+    assert call(src=P + 7 * plane, dst=P, lb=0, le=1) == S.ERR_INVALID_ARG   # source starts in the destination's layer
+    assert call(dst=P + 16, lb=3, le=4, cap=1) == S.ERR_INVALID_ARG          # one row, one layer: still shared bytes
 
 
 def test_kv_compact_rope_rejects_bad_arguments(L):
@@ -160,7 +168,9 @@ def test_kv_compact_rope_rejects_bad_arguments(L):
         base.update(kw)
         return sv.KVLayout(**base)
 
-    def call(src=P, sl=None, dst=2 * P, dl=None, lb=0, le=2, kp=P, kso=P, so=P, B=1, cap=1000, rd=128, rb=1e6,
+    FAR = P + (1 << 40)
+
+    def call(src=P, sl=None, dst=FAR, dl=None, lb=0, le=2, kp=P, kso=P, so=P, B=1, cap=1000, rd=128, rb=1e6,
              ws=P, wsb=1 << 20):
         sl = layout() if sl is None else sl
         dl = layout() if dl is None else dl
@@ -179,6 +189,7 @@ def test_kv_compact_rope_rejects_bad_arguments(L):
     assert call(wsb=64) == S.ERR_WORKSPACE
     assert call(ws=None) == S.ERR_INVALID_ARG
     assert call(lb=1, le=1) == S.OK
+    assert call(dst=P + 4096) == S.ERR_INVALID_ARG                # destination inside the source cache
 
 
 def test_kv_prune_layers_rejects_bad_arguments(L):
