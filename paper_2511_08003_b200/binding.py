@@ -151,6 +151,13 @@ def _check(fn: str, rc: int):
         raise SharpVError(fn, rc)
 
 
+def _call(name: str, on: torch.Tensor, *args) -> int:
+    """Calls the entry point `name` with the device of `on` current: kernels are launched on the current
+    device, and the allocation-free entry point keys its built-in scratch on it."""
+    with torch.cuda.device(on.device):
+        return getattr(lib(), name)(*args)
+
+
 def _workspace(ws: Optional[torch.Tensor], nbytes: int, device) -> torch.Tensor:
     if ws is None:
         return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
@@ -198,7 +205,7 @@ def sharpv_score_frames(tokens: torch.Tensor, video_frame_offsets: torch.Tensor,
         out["temporal"] = torch.empty(n, dtype=torch.float32, device=dev)
     nbytes = sharpv_score_frames_workspace_bytes(total_frames, f, d)
     ws = _workspace(workspace, nbytes, dev)
-    rc = lib().sharpv_score_frames(
+    rc = _call("sharpv_score_frames", tokens,
         _dev(tokens, "tokens"), _dtype_code(tokens), ld, video_frame_offsets.numel() - 1,
         _dev(video_frame_offsets, "video_frame_offsets", torch.int32), total_frames, f, d, float(w),
         int(dissim_kind), int(round_mode), int(min_keep),
@@ -240,10 +247,11 @@ def _select(fn_name, importance, k, K, total_frames, f, tokens, capacity, gather
               _dev(out["num_kept"], "num_kept", torch.int32), ws.data_ptr(), ws.numel(),
               _dev(status_word, "status_word", torch.int32), _stream(stream))
     if fn_name == "sharpv_select_tokens":
-        rc = lib().sharpv_select_tokens(_dev(importance, "importance", torch.float32),
-                                        _dev(k, "k", torch.int32), *common)
+        rc = _call("sharpv_select_tokens", importance, _dev(importance, "importance", torch.float32),
+                   _dev(k, "k", torch.int32), *common)
     else:
-        rc = lib().sharpv_select_tokens_threshold(_dev(importance, "importance", torch.float32), float(K), *common)
+        rc = _call("sharpv_select_tokens_threshold", importance, _dev(importance, "importance", torch.float32),
+                   float(K), *common)
     _check(fn_name, rc)
     return out
 
@@ -296,9 +304,9 @@ def _calibrate(fn_name, hidden, visual, seq_offsets, vis_begin, vis_count, vis_o
     tail = (_dev(status_word, "status_word", torch.int32), _stream(stream))
     if fn_name == "sharpv_kv_calibrate_prune":
         ws = _workspace(workspace, sharpv_kv_calibrate_prune_workspace_bytes(total_seq_tokens, B), dev)
-        rc = lib().sharpv_kv_calibrate_prune(*head, ws.data_ptr(), ws.numel(), *tail)
+        rc = _call("sharpv_kv_calibrate_prune", hidden, *head, ws.data_ptr(), ws.numel(), *tail)
     else:
-        rc = lib().sharpv_kv_calibrate_prune_noalloc(*head, *tail)
+        rc = _call("sharpv_kv_calibrate_prune_noalloc", hidden, *head, *tail)
     _check(fn_name, rc)
     return out
 
@@ -334,7 +342,7 @@ def sharpv_kv_compact(kv_src: torch.Tensor, kv_dst: torch.Tensor, kept_pos: torc
     sl, dl = kv_layout(kv_src), kv_layout(kv_dst)
     if layer_end is None:
         layer_end = kv_src.shape[0]
-    rc = lib().sharpv_kv_compact(
+    rc = _call("sharpv_kv_compact", kv_src,
         _dev(kv_src, "kv_src"), C.byref(sl), _dev(kv_dst, "kv_dst"), C.byref(dl), layer_begin, layer_end,
         _dev(kept_pos, "kept_pos", torch.int32), _dev(kept_seq_offsets, "kept_seq_offsets", torch.int32),
         kept_seq_offsets.numel() - 1, capacity, _dev(status_word, "status_word", torch.int32), _stream(stream))
@@ -370,7 +378,7 @@ def sharpv_kv_prune_layers(hidden_layers: torch.Tensor, visual: torch.Tensor, se
         raise ValueError("sharpv_kv_prune_layers wrapper needs total_visual > 0 and capacity > 0")
     sl, dl = kv_layout(kv_src), kv_layout(kv_dst)
     ws = _workspace(workspace, sharpv_kv_calibrate_prune_workspace_bytes(total_seq_tokens, B), dev)
-    rc = lib().sharpv_kv_prune_layers(
+    rc = _call("sharpv_kv_prune_layers", hidden_layers,
         _dev(hidden_layers, "hidden_layers"), hidden_layers.stride(0), hidden_layers.stride(1),
         _dev(visual, "visual"), ldv, _dtype_code(visual), visual.shape[1], B,
         _dev(seq_offsets, "seq_offsets", torch.int32), _dev(vis_begin, "vis_begin", torch.int32),
@@ -398,7 +406,7 @@ def sharpv_kv_compact_rope(kv_src: torch.Tensor, kv_dst: torch.Tensor, kept_pos:
     if layer_end is None:
         layer_end = kv_src.shape[0]
     ws = _workspace(workspace, sharpv_kv_compact_rope_workspace_bytes(capacity, rotary_dim), kv_src.device)
-    rc = lib().sharpv_kv_compact_rope(
+    rc = _call("sharpv_kv_compact_rope", kv_src,
         _dev(kv_src, "kv_src"), C.byref(sl), _dev(kv_dst, "kv_dst"), C.byref(dl), layer_begin, layer_end,
         _dev(kept_pos, "kept_pos", torch.int32), _dev(kept_seq_offsets, "kept_seq_offsets", torch.int32),
         _dev(seq_offsets, "seq_offsets", torch.int32), kept_seq_offsets.numel() - 1, capacity, int(rotary_dim),

@@ -4,7 +4,8 @@
 // Kernels:
 //   calibrate_cos_kernel  one warp per packed position: cos(hidden row, visual row), keep flag,
 //                         and an integer count of survivors per chunk of 256 positions
-//   write_kept_kernel     (dependent launch) chunk base = sum of earlier chunk counts, local scan,
+//   write_kept_kernel     (dependent launch) chunk base = sum of earlier chunk counts (beyond 4096 chunks a
+//                         one-CTA scan kernel in front turns the counts into bases), local scan,
 //                         ascending kept positions, per-sequence offsets, capacity check
 //   mean_cos_kernel       (optional) fixed-order mean of the cosines of each sequence
 #include <mutex>
@@ -20,6 +21,7 @@ __host__ __device__ inline size_t ws_flags_bytes(int64_t T) { return ((size_t)T 
 __host__ __device__ inline int64_t num_chunks(int64_t T) { return (T + kChunk - 1) / kChunk; }
 
 constexpr int kRowsPerCta = 4;          // one packed position per warp; small CTAs balance the SMs
+constexpr int64_t kInlineBaseChunks = 4096;  // up to this many chunks every chunk CTA adds up the counts in front of it itself
 
 template <int DT>
 __global__ void __launch_bounds__(kRowsPerCta * 32)
@@ -91,7 +93,7 @@ calibrate_cos_kernel(const char* __restrict__ hidden, int64_t hidden_row_bytes,
 }
 
 __global__ void __launch_bounds__(kChunk)
-write_kept_kernel(const uint8_t* __restrict__ flags, const int32_t* __restrict__ chunk_counts,
+write_kept_kernel(const uint8_t* __restrict__ flags, const int32_t* __restrict__ chunk_counts, int bases_ready,
                   int64_t T, int num_seqs, const int32_t* __restrict__ seq_offsets, int64_t capacity,
                   int32_t* __restrict__ out_kept_pos, int32_t* __restrict__ out_kept_seq_offsets,
                   int32_t* status_word) {
@@ -102,8 +104,14 @@ write_kept_kernel(const uint8_t* __restrict__ flags, const int32_t* __restrict__
     // all global loads of this thread are issued up front: one memory round trip, not three
     const int64_t p = (int64_t)c * kChunk + threadIdx.x;
     const int keep = p < T ? flags[p] : 0;
+    // kept positions before this chunk: the counts of the chunks in front, or (many chunks) their
+    // exclusive scan, which a one-CTA kernel in front has left in the same array
     int part = 0;
-    for (int i = threadIdx.x; i < c; i += kChunk) part += chunk_counts[i];
+    if (bases_ready) {
+        if (threadIdx.x == 0) part = chunk_counts[c];
+    } else {
+        for (int i = threadIdx.x; i < c; i += kChunk) part += chunk_counts[i];
+    }
     int seq_first = -1, seq_last = -1;      // sequences that start at p: [seq_first, seq_last]
     if (p < T) {
         int b = upper_segment(seq_offsets, num_seqs, (int)p);
@@ -214,8 +222,16 @@ static sharpv_status calibrate_impl(
             return SHARPV_ERR_CUDA;
         }
     }
+    const int bases_ready = (int64_t)chunks > kInlineBaseChunks;
+    if (bases_ready &&
+        launch_dependent(exclusive_scan_i32_kernel<false>, dim3(1), dim3(kScanThreads), 0, stream,
+                         (const int32_t*)chunk_counts, (int64_t)chunks, 0, chunk_counts, (int32_t*)nullptr,
+                         (int32_t*)nullptr, (int64_t)-1, (int32_t*)nullptr) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SHARPV_ERR_CUDA;
+    }
     if (launch_dependent(write_kept_kernel, dim3(chunks), dim3(kChunk), 0, stream, (const uint8_t*)flags,
-                         (const int32_t*)chunk_counts, total_seq_tokens, num_seqs, seq_offsets, capacity,
+                         (const int32_t*)chunk_counts, bases_ready, total_seq_tokens, num_seqs, seq_offsets, capacity,
                          out_kept_pos, out_kept_seq_offsets, status_word) != cudaSuccess) {
         (void)cudaGetLastError();
         return SHARPV_ERR_CUDA;

@@ -170,4 +170,36 @@ __device__ __forceinline__ void report(int32_t* status_word, int code) {
     if (status_word) atomicMax(status_word, code);
 }
 
+// Exclusive prefix sums of n ints by one CTA of 1024 threads: thread i adds up a contiguous share,
+// one block scan, then every thread writes the prefixes of its share.  out[i] = sum of val(in[j]),
+// j < i, with val = min(max(in[j], 0), clamp_hi) when CLAMP; out == in is allowed.  If out_total is
+// not null it receives the grand total (as do *total_copy, if not null, and the capacity check).
+constexpr int kScanThreads = 1024;
+template <bool CLAMP>
+__global__ void __launch_bounds__(kScanThreads)
+exclusive_scan_i32_kernel(const int32_t* in, int64_t n, int clamp_hi, int32_t* out, int32_t* out_total,
+                          int32_t* total_copy, int64_t capacity, int32_t* status_word) {
+    __shared__ int sm[kScanThreads / 32 + 1];
+    cudaGridDependencySynchronize();
+    const int64_t per = (n + kScanThreads - 1) / kScanThreads;
+    const int64_t lo = min(n, (int64_t)threadIdx.x * per), hi = min(n, lo + per);
+    int sum = 0;
+    for (int64_t i = lo; i < hi; ++i) {
+        const int v = in[i];
+        sum += CLAMP ? min(max(v, 0), clamp_hi) : v;
+    }
+    int total;
+    int run = block_exclusive_scan<kScanThreads>(sum, sm, total);
+    for (int64_t i = lo; i < hi; ++i) {
+        const int v = in[i];
+        out[i] = run;
+        run += CLAMP ? min(max(v, 0), clamp_hi) : v;
+    }
+    if (threadIdx.x == 0) {
+        if (out_total) *out_total = total;
+        if (total_copy) *total_copy = total;
+        if (capacity >= 0 && (int64_t)total > capacity) report(status_word, SHARPV_ERR_CAPACITY);
+    }
+}
+
 }  // namespace sharpv

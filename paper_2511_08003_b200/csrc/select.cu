@@ -4,7 +4,8 @@
 //
 // Kernels:
 //   count_above_kernel   (threshold variant only) per-frame count of I > K
-//   select_frame_kernel  one CTA per frame: its offset (sum of the budgets in front of it), then in
+//   select_frame_kernel  one CTA per frame: its offset (sum of the budgets in front of it; beyond 4096
+//                        frames a one-CTA scan kernel in front computes all offsets), then in
 //                        shared memory either a rank count over composite (key, index) keys (frames
 //                        of up to 1024 tokens) or a 4-pass byte radix select of the k-th largest key
 //                        with an index-ordered scan for the tie-break; ascending indices out
@@ -18,6 +19,7 @@ namespace {
 constexpr int kSelectThreads = 256;
 constexpr int kMaxTokensPerFrame = 8192;
 constexpr int kRankMaxTokens = 1024;     // frames up to this size are selected by counting ranks
+constexpr int kInlineOffsetFrames = 4096; // up to this many frames every frame CTA adds up the budgets in front of it itself
 
 // Monotone map fp32 -> uint32: larger score, larger key.  Adding +0 turns -0 into +0.
 __device__ __forceinline__ uint32_t order_key(float x) {
@@ -44,7 +46,7 @@ count_above_kernel(const float* __restrict__ importance, float K, int f, int32_t
 // mode 0: top-k with budgets k[t];  mode 1: keep I > K
 __global__ void __launch_bounds__(kSelectThreads)
 select_frame_kernel(const float* __restrict__ importance, const int32_t* __restrict__ k, int F, int f,
-                    int64_t capacity, int mode, float K, int32_t* __restrict__ kept_offsets,
+                    int64_t capacity, int mode, float K, int offsets_ready, int32_t* __restrict__ kept_offsets,
                     int32_t* __restrict__ num_kept, int32_t* __restrict__ out_kept_index, int32_t* status_word) {
     extern __shared__ __align__(16) uint32_t keys[];   // [f]
     __shared__ int hist[4][256];                       // one histogram per byte pass, cleared once
@@ -58,8 +60,10 @@ select_frame_kernel(const float* __restrict__ importance, const int32_t* __restr
     cudaGridDependencySynchronize();        // scores and budgets come from earlier work on the stream
 
     // this frame's offset: the (clamped) budgets of the frames in front of it, added in a fixed order
+    // here, or read from the scan a kernel in front has left in kept_offsets (large batches)
     int part = 0;
-    for (int i = tid; i < t; i += kSelectThreads) part += min(max(k[i], 0), f);
+    if (!offsets_ready)
+        for (int i = tid; i < t; i += kSelectThreads) part += min(max(k[i], 0), f);
     const int kt_raw = k[t];
     for (int i = tid; i < f; i += kSelectThreads) keys[i] = mode == 0 ? order_key(imp[i]) : (imp[i] > K ? 1u : 0u);
     for (int i = tid; i < 4 * 256; i += kSelectThreads) (&hist[0][0])[i] = 0;
@@ -67,10 +71,14 @@ select_frame_kernel(const float* __restrict__ importance, const int32_t* __restr
     if (lane == 0) off_sm[warp] = part;
     __syncthreads();
     int before = 0;
+    if (offsets_ready) {
+        before = kept_offsets[t];
+    } else {
 #pragma unroll
-    for (int i = 0; i < kSelectThreads / 32; ++i) before += off_sm[i];
+        for (int i = 0; i < kSelectThreads / 32; ++i) before += off_sm[i];
+    }
     const int64_t out_base = before;
-    if (tid == 0) {
+    if (tid == 0 && !offsets_ready) {
         kept_offsets[t] = before;
         if (t == F - 1) {
             const int total = before + min(max(kt_raw, 0), f);
@@ -249,9 +257,17 @@ sharpv_status select_impl(int mode, const float* importance, const int32_t* k, f
     }
     // keys, plus the 64-bit composite keys of the rank-counting path for small frames
     const size_t sel_smem = (size_t)((f + 3) & ~3) * 4 + (f <= kRankMaxTokens ? (size_t)((f + 1) & ~1) * 8 : 0);
+    const int offsets_ready = F > kInlineOffsetFrames;
+    if (offsets_ready &&
+        launch_dependent(exclusive_scan_i32_kernel<true>, dim3(1), dim3(kScanThreads), 0, stream, budgets, (int64_t)F,
+                         (int)f, out_kept_offsets, out_kept_offsets + F, out_num_kept, capacity, status_word) !=
+            cudaSuccess) {
+        (void)cudaGetLastError();
+        return SHARPV_ERR_CUDA;
+    }
     if (launch_dependent(select_frame_kernel, dim3((unsigned)F), dim3(kSelectThreads), sel_smem, stream,
-                         importance, budgets, (int)F, (int)f, capacity, mode, K, out_kept_offsets, out_num_kept,
-                         out_kept_index, status_word) != cudaSuccess) {
+                         importance, budgets, (int)F, (int)f, capacity, mode, K, offsets_ready, out_kept_offsets,
+                         out_num_kept, out_kept_index, status_word) != cudaSuccess) {
         (void)cudaGetLastError();
         return SHARPV_ERR_CUDA;
     }

@@ -721,6 +721,63 @@ def test_stage_two_random_layouts(seed):
     assert store == got.dtype
 
 
+def test_many_frames_and_many_positions_use_the_scan_kernels():
+    """Batches beyond the sizes at which every CTA adds up the counts in front of it itself: 20,000 tiny
+    frames through the selection, 1.2 million packed positions through the calibration (their offsets then
+    come from the one-CTA scan kernel)."""
+    rng = np.random.default_rng(77)
+    F, f = 20_000, 5
+    imp = rng.random(F * f).astype(np.float32)
+    imp[rng.integers(0, F * f, 3000)] = 0.5                        # ties
+    k = rng.integers(-1, f + 2, F).astype(np.int32)                # budgets outside [0, f] are clamped
+    sel = sv.sharpv_select_tokens(to_dev(imp), to_dev(k), F, f, gather=False)
+    torch.cuda.synchronize()
+    idx_o, off_o = orc.select_tokens(imp, k, f)
+    np.testing.assert_array_equal(to_host(sel["kept_offsets"]), off_o)
+    assert int(sel["num_kept"].item()) == idx_o.size
+    np.testing.assert_array_equal(to_host(sel["kept_index"])[:idx_o.size], idx_o)
+    thr = sv.sharpv_select_tokens_threshold(to_dev(imp), 0.5, F, f, gather=False)
+    torch.cuda.synchronize()
+    idx_t, off_t = orc.select_threshold(imp, 0.5, F, f)
+    np.testing.assert_array_equal(to_host(thr["kept_offsets"]), off_t)
+    np.testing.assert_array_equal(to_host(thr["kept_index"])[:idx_t.size], idx_t)
+    # capacity overflow is still reported by the scan
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    small = sv.sharpv_select_tokens(to_dev(imp), to_dev(k), F, f, gather=False, capacity=100, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == sv.Status.ERR_CAPACITY and int(small["num_kept"].item()) == idx_o.size
+    np.testing.assert_array_equal(to_host(small["kept_index"])[:100], idx_o[:100])
+
+    T, d = 1_200_000, 16
+    lens = np.array([400_000, 0, 799_990, 10])
+    so = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    vb = np.array([5, 0, 1000, 0], np.int32)
+    vc = np.array([300_000, 0, 500_000, 10], np.int32)
+    vo = np.concatenate([[0], np.cumsum(vc)])[:-1].astype(np.int32)
+    vis = rng.standard_normal((int(vc.sum()), d)).astype(np.float32)
+    hid = rng.standard_normal((T, d)).astype(np.float32)
+    for b in range(4):
+        r0 = so[b] + vb[b]
+        hid[r0:r0 + vc[b]] += 1.5 * vis[vo[b]:vo[b] + vc[b]]
+    t32 = lambda a: torch.from_numpy(np.asarray(a, np.int32)).cuda()
+    g = sv.sharpv_kv_calibrate_prune(to_dev(hid), to_dev(vis), t32(so), t32(vb), t32(vc), t32(vo), T, M=0.8)
+    torch.cuda.synchronize()
+    o = orc.kv_calibrate_prune(hid, vis, so, vb, vc, vo, 0.8, nthreads=NT)
+    assert rel_err(to_host(g["cos"]), o["cos"]) <= TIGHT_TOL
+    kso = to_host(g["kept_seq_offsets"])
+    kept = to_host(g["kept_pos"])[:kso[-1]]
+    assert np.all(np.diff(kept) > 0)
+    sym = np.setxor1d(kept, o["kept_pos"])
+    for pos in sym:                                                 # only cosines at the threshold may differ
+        b = int(np.searchsorted(so, pos, side="right") - 1)
+        row = vo[b] + (pos - so[b] - vb[b])
+        assert 0 <= pos - so[b] - vb[b] < vc[b] and abs(o["cos"][row] - 0.8) <= BOUNDARY_TOL
+    assert sym.size <= 20
+    if sym.size == 0:
+        np.testing.assert_array_equal(kso, o["kept_seq_offsets"])
+    assert 0.2 * T < kept.size < 0.9 * T
+
+
 def test_run_to_run_bit_reproducible():
     wl, dw = _case("small_ragged")
     F, f = wl.total_frames, wl.f

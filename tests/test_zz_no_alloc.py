@@ -15,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import sharpv_oracle as orc
 from paper_2511_08003_b200 import binding as sv
 from paper_2511_08003_b200 import workloads as W
 
@@ -64,6 +65,20 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
         torch.cuda.synchronize()
         kept.append(_same(got, ref, wl.n_visual))
         assert 0 < kept[-1] < wl.total_seq_tokens            # the threshold actually prunes something
+        # and against the CPU oracle directly, so that this file stands on its own
+        o = orc.kv_calibrate_prune(wl.hidden, wl.tokens, wl.seq_offsets, wl.vis_begin, wl.vis_count, wl.vis_offsets,
+                                   M, nthreads=4)
+        cos = got["cos"].cpu().numpy().astype(np.float64)
+        assert np.max(np.abs(cos - o["cos"])) <= 1e-5
+        away = np.abs(o["cos"] - M) > 1e-5                    # tokens whose oracle cosine is not at the threshold
+        pos = np.concatenate([wl.seq_offsets[b] + wl.vis_begin[b] + np.arange(wl.vis_count[b])
+                              for b in range(wl.num_videos)])
+        mine = np.zeros(wl.total_seq_tokens, bool)
+        mine[got["kept_pos"][:kept[-1]].cpu().numpy()] = True
+        theirs = np.zeros(wl.total_seq_tokens, bool)
+        theirs[o["kept_pos"]] = True
+        assert np.array_equal(mine[pos][away], theirs[pos][away])
+        assert np.array_equal(np.delete(mine, pos), np.delete(theirs, pos))      # text positions: all kept
     assert int(status.item()) == 0
     # and once more on the first input: the scratch now holds the small call's leftovers
     args = _inputs(big, dev)
@@ -71,6 +86,34 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
     got = sv.sharpv_kv_calibrate_prune_noalloc(*args, M=0.788, want_mean_cos=True, out=_outputs(big, dev))
     torch.cuda.synchronize()
     assert _same(got, ref, big.n_visual) == kept[0]
+
+
+def test_noalloc_takes_the_largest_input_it_documents_and_allocates_nothing():
+    """total_seq_tokens == SHARPV_NOALLOC_MAX_SEQ_TOKENS uses the fixed scratch to its last byte; with all
+    outputs passed in, the device's free memory is the same before and after the call."""
+    dev = torch.device("cuda", 0)
+    T, d, n_vis = sv.NOALLOC_MAX_SEQ_TOKENS, 64, 200_000
+    g = torch.Generator(device=dev)
+    g.manual_seed(62)
+    visual = torch.randn((n_vis, d), dtype=torch.float32, device=dev, generator=g)
+    hidden = torch.randn((T, d), dtype=torch.float32, device=dev, generator=g)
+    hidden[1000:1000 + n_vis] = visual + 0.9 * hidden[1000:1000 + n_vis]
+    i32 = lambda v: torch.tensor(v, dtype=torch.int32, device=dev)
+    tabs = (i32([0, T]), i32([1000]), i32([n_vis]), i32([0]))
+    ref = sv.sharpv_kv_calibrate_prune(hidden, visual, *tabs, T, M=0.75, want_mean_cos=True)
+    out = {"cos": torch.empty(n_vis, dtype=torch.float32, device=dev),
+           "kept_pos": torch.empty(T, dtype=torch.int32, device=dev),
+           "kept_seq_offsets": torch.empty(2, dtype=torch.int32, device=dev),
+           "mean_cos": torch.empty(1, dtype=torch.float32, device=dev)}
+    sv.sharpv_kv_calibrate_prune_noalloc(hidden, visual, *tabs, T, M=0.75, want_mean_cos=True, out=out)   # set-up call
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info(dev)
+    got = sv.sharpv_kv_calibrate_prune_noalloc(hidden, visual, *tabs, T, M=0.75, want_mean_cos=True, out=out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info(dev)
+    assert free_after == free_before
+    n = _same(got, ref, n_vis)
+    assert T - n_vis < n < T
 
 
 def test_noalloc_rejects_inputs_beyond_its_fixed_scratch():
