@@ -4,7 +4,7 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl sharpv|reference]
 
 One "step" is one pass of the whole path over one batch of synthetic video tokens:
-score frames -> per-frame top-k + gather -> calibration -> K/V compaction.  Prints one JSON
+stage one in one call (scores, budgets, per-frame top-k, gather) -> calibration -> K/V compaction.  Prints one JSON
 line (rank 0).  With N > 1 every rank runs the same-shaped batch on its own GPU (videos are
 independent: no data-path collective, weak scaling) and the time is the max over ranks.
 `--impl reference` times the CPU oracle on the host cores instead.
@@ -37,9 +37,10 @@ NOMINAL_HBM_GBS = 8000.0
 MIN_TIMED_SECONDS = 0.3
 KERNEL_REPLAYS = 20
 REPORTED_WORKLOADS = ("onevision_7b", "video_7b", "ragged_batch", "long_video")
-STAGES = ("score", "select", "calibrate", "compact")
-# kernels launched per step by each entry point (score, select, calibrate, compact)
-LAUNCHES_PER_STEP = {"score": 2, "select": 2, "calibrate": 2, "compact": 1}
+STEP_STAGES = ("prune", "calibrate", "compact")                    # the entry points one step calls
+STAGES = ("prune", "score", "select", "calibrate", "compact")      # the entry points that are timed one by one
+# kernels launched by each entry point
+LAUNCHES_PER_STEP = {"prune": 3, "score": 2, "select": 2, "calibrate": 2, "compact": 1}
 # DRAM read + write bytes of one launch of an entry point's main kernel, from ncu captures.  An entry is
 # used only when the run reproduces the captured launch (same workload, threshold, kept count, plain
 # out-of-place compaction); `commit` is the source revision the counters were taken on.
@@ -91,6 +92,9 @@ def algorithmic_bytes(wl, n_keep_tokens, t_keep, stage):
         return wl.n_visual * wl.d * e + wl.n_visual * 4 + wl.total_frames * 8
     if stage == "select":
         return wl.n_visual * 4 + wl.total_frames * 4 + 2 * n_keep_tokens * wl.d * e + n_keep_tokens * 4
+    if stage == "prune":        # stage one in one call: the scores are written but not read back
+        return (wl.n_visual * wl.d * e + wl.n_visual * 4 + wl.total_frames * 8 +
+                2 * n_keep_tokens * wl.d * e + n_keep_tokens * 4)
     if stage == "calibrate":
         return 2 * wl.n_visual * wl.d * e + wl.n_visual * 4 + t_keep * 4
     if stage == "compact":
@@ -320,6 +324,8 @@ class DevicePath:
                       "num_kept": torch.empty(1, dtype=torch.int32, device=dev),
                       "tokens": torch.empty((NV, d), dtype=tdt, device=dev)}
         self.ws_sel = torch.empty(sv.sharpv_select_tokens_workspace_bytes(F, f), dtype=torch.uint8, device=dev)
+        self.o_prune = dict(self.o_score, **self.o_sel)
+        self.ws_prune = torch.empty(sv.sharpv_prune_frames_workspace_bytes(F, f, d), dtype=torch.uint8, device=dev)
         self.o_cal = {"cos": torch.empty(NV, dtype=torch.float32, device=dev),
                       "kept_pos": torch.empty(T, dtype=torch.int32, device=dev),
                       "kept_seq_offsets": torch.empty(wl.num_videos + 1, dtype=torch.int32, device=dev)}
@@ -327,9 +333,15 @@ class DevicePath:
                                   device=dev)
         self.ws_rope = (torch.empty(sv.sharpv_kv_compact_rope_workspace_bytes(T, wl.head_dim), dtype=torch.uint8,
                                     device=dev) if args.rope else None)
-        self.stages = {"score": self.stage_score, "select": self.stage_select, "calibrate": self.stage_calibrate,
-                       "compact": self.stage_compact}
+        self.stages = {"prune": self.stage_prune, "score": self.stage_score, "select": self.stage_select,
+                       "calibrate": self.stage_calibrate, "compact": self.stage_compact}
         self.n_keep = self.t_keep = None
+
+    def stage_prune(self, i=0):
+        wl = self.wl
+        self.sv.sharpv_prune_frames(self.tok_copies[i % self.ncopies], self.tabs["video_frame_offsets"],
+                                    wl.total_frames, wl.f, w=self.args.w, capacity=wl.n_visual, out=self.o_prune,
+                                    workspace=self.ws_prune, status_word=self.status)
 
     def stage_score(self, i=0):
         wl = self.wl
@@ -362,7 +374,7 @@ class DevicePath:
                                   capacity=T, status_word=self.status)
 
     def step(self):
-        for name in STAGES:
+        for name in STEP_STAGES:
             self.stages[name]()
 
     def warm(self, n):
@@ -608,7 +620,7 @@ def run_sharpv(args):
             dist.destroy_process_group()
         return
 
-    dom = max(STAGES, key=lambda k: kernels[k]["median_ms"])
+    dom = max(STEP_STAGES, key=lambda k: kernels[k]["median_ms"])
     cap = NCU_TRAFFIC.get((args.workload, dom))
     same_launch = (cap is not None and not args.inplace and not args.rope and args.frames is None and
                    args.layers is None and abs(cap["M"] - args.M) < 1e-9 and cap["kept_stage_two"] == t_keep)
@@ -673,7 +685,7 @@ def run_sharpv(args):
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "note": "tokens and hidden state copied from pinned host memory every step, kept-index lists "
                         "read back; the K/V cache is device-resident model state"},
-        "gpu_launches": sum(LAUNCHES_PER_STEP.values()) * replays,
+        "gpu_launches": sum(LAUNCHES_PER_STEP[k] for k in STEP_STAGES) * replays,
         "clocks": clocks, "wall_s": round(wall, 3),
     }
     print(json.dumps(line))

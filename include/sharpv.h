@@ -137,6 +137,29 @@ sharpv_status sharpv_select_tokens_threshold(
     void* workspace, size_t workspace_bytes, int32_t* status_word, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Stage one in one call.  Section 3.1 describes Visual SharpV as one pipeline: importance scores, from
+ * them the retention ratio of every frame, and the retention of each frame's highest-scoring tokens.
+ * sharpv_prune_frames computes exactly what sharpv_score_frames followed by sharpv_select_tokens (with
+ * the budgets out_k) computes, and writes the same outputs, but the selection runs where the frame's
+ * scores are produced: the scores are not read back from memory and two launches fall away.
+ * Arguments as in those two entry points; workspace of sharpv_prune_frames_workspace_bytes() bytes,
+ * 256-byte aligned.  f <= 8192; frames of more than 256 tokens and rows that are not a multiple of 128
+ * bytes run the two entry points one after the other inside the call.
+ */
+size_t sharpv_prune_frames_workspace_bytes(int32_t total_frames, int32_t f, int32_t d);
+
+sharpv_status sharpv_prune_frames(
+    const void* tokens, sharpv_dtype dtype, int64_t ld_tokens,
+    int32_t num_videos, const int32_t* video_frame_offsets, int32_t total_frames,
+    int32_t f, int32_t d,
+    float w, sharpv_dissim_kind dissim_kind, sharpv_round round_mode, int32_t min_keep,
+    float* out_importance, float* out_spatial, float* out_temporal,
+    float* out_ratio, int32_t* out_k,
+    int32_t* out_kept_index, int32_t* out_kept_offsets,
+    void* out_tokens, int64_t capacity, int32_t* out_num_kept,
+    void* workspace, size_t workspace_bytes, int32_t* status_word, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
  * Stage two (a): self-calibration.  Section 3.2.3, Eq. 7, applied per visual token.
  *
  * hidden [dev] [total_seq_tokens, d]: the hidden state G_l of the chosen layer for all

@@ -53,6 +53,7 @@ EXPORTS = (
     "sharpv_version", "sharpv_status_string",
     "sharpv_score_frames_workspace_bytes", "sharpv_score_frames",
     "sharpv_select_tokens_workspace_bytes", "sharpv_select_tokens", "sharpv_select_tokens_threshold",
+    "sharpv_prune_frames_workspace_bytes", "sharpv_prune_frames",
     "sharpv_kv_calibrate_prune_workspace_bytes", "sharpv_kv_calibrate_prune",
     "sharpv_kv_calibrate_prune_noalloc",
     "sharpv_kv_prune_layers", "sharpv_kv_compact",
@@ -92,6 +93,11 @@ def lib():
     L.sharpv_select_tokens_threshold.restype = C.c_int
     L.sharpv_select_tokens_threshold.argtypes = [vp, f32, i32, i32, vp, C.c_int, i64, i32, vp, vp, vp, i64, vp,
                                                  vp, sz, vp, vp]
+    L.sharpv_prune_frames_workspace_bytes.restype = sz
+    L.sharpv_prune_frames_workspace_bytes.argtypes = [i32, i32, i32]
+    L.sharpv_prune_frames.restype = C.c_int
+    L.sharpv_prune_frames.argtypes = [vp, C.c_int, i64, i32, vp, i32, i32, i32, f32, C.c_int, C.c_int, i32,
+                                      vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp, vp]
     L.sharpv_kv_calibrate_prune_workspace_bytes.restype = sz
     L.sharpv_kv_calibrate_prune_workspace_bytes.argtypes = [i64, i32]
     L.sharpv_kv_calibrate_prune.restype = C.c_int
@@ -270,6 +276,55 @@ def sharpv_select_tokens_threshold(importance: torch.Tensor, K: float, total_fra
     """Manual variant: keep importance > K.  Same outputs as sharpv_select_tokens."""
     return _select("sharpv_select_tokens_threshold", importance, None, K, total_frames, f, tokens, capacity,
                    gather and tokens is not None, out, workspace, status_word, stream)
+
+
+def sharpv_prune_frames_workspace_bytes(total_frames: int, f: int, d: int) -> int:
+    return int(lib().sharpv_prune_frames_workspace_bytes(total_frames, f, d))
+
+
+def sharpv_prune_frames(tokens: torch.Tensor, video_frame_offsets: torch.Tensor, total_frames: int, f: int,
+                        w: float = 1.0, dissim_kind: int = DISSIM, round_mode: int = ROUND_FLOOR,
+                        min_keep: int = 0, want_spatial: bool = False, want_temporal: bool = False,
+                        capacity: Optional[int] = None, gather: bool = True,
+                        out: Optional[Dict[str, torch.Tensor]] = None, workspace: Optional[torch.Tensor] = None,
+                        status_word: Optional[torch.Tensor] = None, stream=None) -> Dict[str, torch.Tensor]:
+    """Stage one in one call: the outputs of sharpv_score_frames and of sharpv_select_tokens run on its
+    budgets.  Returns dict(importance, ratio, k, kept_index, kept_offsets, num_kept[, tokens, spatial,
+    temporal])."""
+    ld = _rows(tokens, "tokens")
+    d = tokens.shape[1]
+    dev = tokens.device
+    out = dict(out) if out else {}
+    n = total_frames * f
+    if capacity is None:
+        capacity = n
+    new = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
+    out.setdefault("importance", new(n, torch.float32))
+    out.setdefault("ratio", new(total_frames, torch.float32))
+    out.setdefault("k", new(total_frames, torch.int32))
+    if want_spatial:
+        out.setdefault("spatial", new(n, torch.float32))
+    if want_temporal:
+        out.setdefault("temporal", new(n, torch.float32))
+    out.setdefault("kept_index", new(max(capacity, 1), torch.int32))
+    out.setdefault("kept_offsets", new(total_frames + 1, torch.int32))
+    out.setdefault("num_kept", new(1, torch.int32))
+    if gather:
+        out.setdefault("tokens", new((max(capacity, 1), d), tokens.dtype))
+    ws = _workspace(workspace, sharpv_prune_frames_workspace_bytes(total_frames, f, d), dev)
+    rc = _call("sharpv_prune_frames", tokens,
+               _dev(tokens, "tokens"), _dtype_code(tokens), ld, video_frame_offsets.numel() - 1,
+               _dev(video_frame_offsets, "video_frame_offsets", torch.int32), total_frames, f, d, float(w),
+               int(dissim_kind), int(round_mode), int(min_keep),
+               _dev(out["importance"], "importance", torch.float32), _dev(out.get("spatial"), "spatial", torch.float32),
+               _dev(out.get("temporal"), "temporal", torch.float32), _dev(out["ratio"], "ratio", torch.float32),
+               _dev(out["k"], "k", torch.int32), _dev(out["kept_index"], "kept_index", torch.int32),
+               _dev(out["kept_offsets"], "kept_offsets", torch.int32),
+               _dev(out.get("tokens"), "out tokens") if gather else None, capacity,
+               _dev(out["num_kept"], "num_kept", torch.int32), ws.data_ptr(), ws.numel(),
+               _dev(status_word, "status_word", torch.int32), _stream(stream))
+    _check("sharpv_prune_frames", rc)
+    return out
 
 
 def sharpv_kv_calibrate_prune_workspace_bytes(total_seq_tokens: int, num_seqs: int) -> int:

@@ -166,6 +166,22 @@ __device__ __forceinline__ int upper_segment(const int32_t* __restrict__ offsets
     return lo;
 }
 
+// same search on a table any address space may hold (shared memory copies of an offset table)
+__device__ __forceinline__ int upper_segment_any(const int32_t* offsets, int n, int x) {
+    int lo = 0, hi = n;
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (offsets[mid] <= x) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// Monotone map fp32 -> uint32: larger score, larger key.  Adding +0 turns -0 into +0.
+__device__ __forceinline__ uint32_t order_key(float x) {
+    const uint32_t b = __float_as_uint(x + 0.0f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
 __device__ __forceinline__ void report(int32_t* status_word, int code) {
     if (status_word) atomicMax(status_word, code);
 }

@@ -235,6 +235,8 @@ extern "C" sharpv_status sharpv_score_frames(
         a.one_minus_cos = omc; a.round_mode = (int)round_mode; a.min_keep = min_keep;
         a.out_I = out_importance; a.out_S = out_spatial; a.out_T = out_temporal; a.out_ratio = out_ratio;
         a.out_k = out_k; a.workspace = workspace; a.status_word = status_word; a.stream = stream;
+        a.select = false; a.out_kept_index = nullptr; a.out_kept_offsets = nullptr; a.out_num_kept = nullptr;
+        a.out_tokens = nullptr; a.capacity = 0;
         const sharpv_status st = fused_score_launch(a);
         if (st != SHARPV_ERR_UNSUPPORTED) return st;      // otherwise: set-up unavailable, use the generic kernels
     }
@@ -251,4 +253,75 @@ extern "C" sharpv_status sharpv_score_frames(
     return launch_score<SHARPV_BF16>(tokens, ld_tokens, num_videos, video_frame_offsets, total_frames, f, d, w,
                                      omc, (int)round_mode, min_keep, out_importance, out_spatial, out_temporal,
                                      out_ratio, out_k, ws, stream);
+}
+
+
+// ---------------------------------------------------------------------------------------
+// Stage one in one call (Section 3.1): scores, budgets, per-frame top-k, gather.
+// ---------------------------------------------------------------------------------------
+namespace {
+size_t prune_fused_bytes(int32_t F, int32_t f, int32_t d) {
+    return fused_score_workspace_bytes(F, f, d) + fused_select_workspace_bytes(F, f);
+}
+}  // namespace
+
+extern "C" size_t sharpv_prune_frames_workspace_bytes(int32_t total_frames, int32_t f, int32_t d) {
+    if (total_frames <= 0 || f <= 0 || d <= 0) return 256;
+    const size_t parts = sharpv_score_frames_workspace_bytes(total_frames, f, d) +
+                         sharpv_select_tokens_workspace_bytes(total_frames, f);
+    const size_t fused = prune_fused_bytes(total_frames, f, d);
+    return parts > fused ? parts : fused;
+}
+
+extern "C" sharpv_status sharpv_prune_frames(
+    const void* tokens, sharpv_dtype dtype, int64_t ld_tokens, int32_t num_videos,
+    const int32_t* video_frame_offsets, int32_t total_frames, int32_t f, int32_t d, float w,
+    sharpv_dissim_kind dissim_kind, sharpv_round round_mode, int32_t min_keep, float* out_importance,
+    float* out_spatial, float* out_temporal, float* out_ratio, int32_t* out_k, int32_t* out_kept_index,
+    int32_t* out_kept_offsets, void* out_tokens, int64_t capacity, int32_t* out_num_kept, void* workspace,
+    size_t workspace_bytes, int32_t* status_word, void* cuda_stream) {
+    if (!dtype_ok(dtype)) return SHARPV_ERR_UNSUPPORTED;
+    if (num_videos < 1 || total_frames < 0 || f < 1 || d < 1 || min_keep < 0 || ld_tokens < d || capacity < 0)
+        return SHARPV_ERR_INVALID_ARG;
+    if ((int)round_mode < 0 || (int)round_mode > 2 || (int)dissim_kind < 0 || (int)dissim_kind > 1)
+        return SHARPV_ERR_INVALID_ARG;
+    if (!video_frame_offsets || !out_kept_offsets) return SHARPV_ERR_INVALID_ARG;
+    if (capacity > 0 && !out_kept_index) return SHARPV_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (total_frames == 0) {
+        if (cudaMemsetAsync(out_kept_offsets, 0, sizeof(int32_t), stream) != cudaSuccess) return SHARPV_ERR_CUDA;
+        if (out_num_kept && cudaMemsetAsync(out_num_kept, 0, sizeof(int32_t), stream) != cudaSuccess)
+            return SHARPV_ERR_CUDA;
+        return SHARPV_OK;
+    }
+    if (!tokens || !out_importance || !out_ratio || !out_k || !workspace) return SHARPV_ERR_INVALID_ARG;
+    if ((int64_t)total_frames * f >= (int64_t)1 << 31) return SHARPV_ERR_UNSUPPORTED;
+    const int eb = elem_bytes(dtype);
+    if (((int64_t)d * eb) % 16 || (ld_tokens * eb) % 16 || !aligned16(tokens) || !aligned16(workspace) ||
+        (out_tokens && !aligned16(out_tokens)))
+        return SHARPV_ERR_UNSUPPORTED;
+    if (workspace_bytes < sharpv_prune_frames_workspace_bytes(total_frames, f, d)) return SHARPV_ERR_WORKSPACE;
+
+    if (fused_score_supported(dtype, f, d)) {
+        FusedScoreArgs a;
+        a.tokens = tokens; a.dtype = dtype; a.ld_tokens = ld_tokens; a.num_videos = num_videos;
+        a.video_frame_offsets = video_frame_offsets; a.F = total_frames; a.f = f; a.d = d; a.w = w;
+        a.one_minus_cos = dissim_kind == SHARPV_ONE_MINUS_COS; a.round_mode = (int)round_mode; a.min_keep = min_keep;
+        a.out_I = out_importance; a.out_S = out_spatial; a.out_T = out_temporal; a.out_ratio = out_ratio;
+        a.out_k = out_k; a.workspace = workspace; a.status_word = status_word; a.stream = stream;
+        a.select = true; a.out_kept_index = out_kept_index; a.out_kept_offsets = out_kept_offsets;
+        a.out_num_kept = out_num_kept; a.out_tokens = out_tokens; a.capacity = capacity;
+        const sharpv_status st = fused_score_launch(a);
+        if (st != SHARPV_ERR_UNSUPPORTED) return st;      // otherwise: set-up unavailable, run the two entry points
+    }
+    // shapes outside the fused kernels: the two entry points one after the other
+    const size_t score_bytes = sharpv_score_frames_workspace_bytes(total_frames, f, d);
+    sharpv_status st = sharpv_score_frames(tokens, dtype, ld_tokens, num_videos, video_frame_offsets, total_frames, f, d,
+                                           w, dissim_kind, round_mode, min_keep, out_importance, out_spatial,
+                                           out_temporal, out_ratio, out_k, workspace, score_bytes, status_word,
+                                           cuda_stream);
+    if (st != SHARPV_OK) return st;
+    return sharpv_select_tokens(out_importance, out_k, total_frames, f, tokens, dtype, ld_tokens, d, out_kept_index,
+                                out_kept_offsets, out_tokens, capacity, out_num_kept, (char*)workspace + score_bytes,
+                                workspace_bytes - score_bytes, status_word, cuda_stream);
 }

@@ -41,6 +41,16 @@ __device__ __forceinline__ float dissim_sq_from_dot(float saa, float sbb, float 
 constexpr float kRefineBelowDot = 6.25e-2f;
 
 
+// a * ca - b * cb with a single rounding of the difference: p = fl(a ca), e = a ca - p exactly (one
+// fma), fl(p - b cb) by a second fma, then the exact error back in.  For nearly parallel rows the
+// two products cancel to a few units in their last place; a plain fma(a, ca, -fl(b cb)) would
+// leave the rounding of fl(b cb), which is as large as the difference itself.
+__device__ __forceinline__ float scaled_difference(float a, float ca, float b, float cb) {
+    const float p = a * ca;
+    const float e = fmaf(a, ca, -p);
+    return fmaf(-b, cb, p) + e;
+}
+
 // Exact re-evaluation of one token row: sums the squared differences of the normalised rows
 // directly.  One warp per row; every lane returns the warp totals.  ia, ib, im are the
 // reciprocal (clamped) norms of the row, of the previous-frame row and of the frame mean.
@@ -62,7 +72,7 @@ __device__ __forceinline__ void refine_row(const char* pa, const char* pb, const
             }
 #pragma unroll
             for (int j = 0; j < P; ++j) {
-                const float df = fmaf(a[j], ia, -m[j] * im);
+                const float df = scaled_difference(a[j], ia, m[j], im);
                 es = fmaf(df, df, es);
             }
         }
@@ -70,7 +80,7 @@ __device__ __forceinline__ void refine_row(const char* pa, const char* pb, const
             E::widen(ld_cached(pb + (int64_t)v * 16), b);
 #pragma unroll
             for (int j = 0; j < P; ++j) {
-                const float df = fmaf(a[j], ia, -b[j] * ib);
+                const float df = scaled_difference(a[j], ia, b[j], ib);
                 et = fmaf(df, df, et);
             }
         }

@@ -49,6 +49,7 @@ struct FusedParams {
     float* mean;            // [F, d]
     float4* part;           // [F, nsl, f]: (||a||^2, <a, mean>, ||a-b||^2, ||b||^2) of the row's part in the slice,
                             // b = the same position one frame earlier
+    int32_t* kept_local;    // [F, f] or null: the finaliser also selects; frame t's kept tokens (ascending) at t * f
     int W;                  // warps per CTA: a tile is covered in R = ceil(f / 4W) visits
 };
 
@@ -380,7 +381,7 @@ score_finalize_kernel(const FusedParams p) {
     __shared__ float4 g_sum[4][kMaxTokensFused];
     __shared__ float f_s2[kMaxTokensFused], f_t2[kMaxTokensFused], f_aa[kMaxTokensFused], f_bb[kMaxTokensFused];
     __shared__ int f_fl[kMaxTokensFused];
-    __shared__ float red[kFinThreads / 32];
+    __shared__ float red[kFinThreads / 32 + 1];     // also the scratch of the block scan
     const int t = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row = tid & (kMaxTokensFused - 1), grp = tid >> 8;
@@ -446,10 +447,11 @@ score_finalize_kernel(const FusedParams p) {
         }
     }
     __syncthreads();
-    float tsq = 0.f;
+    float tsq = 0.f, my_I = 0.f;
     if (tid < p.f) {
         float S, T, I;
         scores_from_sq(f_s2[tid], f_t2[tid], is_first, p.one_minus_cos, p.w, S, T, I);
+        my_I = I;
         const int64_t o = (int64_t)t * p.f + tid;
         p.out_I[o] = I;
         if (p.out_S) p.out_S[o] = S;
@@ -464,8 +466,106 @@ score_finalize_kernel(const FusedParams p) {
 #pragma unroll
         for (int i = 0; i < kFinThreads / 32; ++i) tot += red[i];
         const float r = ratio_from_sumsq(tot, p.f);
+        const int kt = budget_from_ratio(r, p.f, p.round_mode, p.min_keep);
         p.out_ratio[t] = r;
-        p.out_k[t] = budget_from_ratio(r, p.f, p.round_mode, p.min_keep);
+        p.out_k[t] = kt;
+        f_fl[0] = kt;
+    }
+    if (!p.kept_local) return;
+
+    // Per-frame top-k (Section 3.1.3, last paragraph) while the frame's scores are still here: a token's
+    // rank under (score descending, index ascending) is the number of composite (key, ~index) keys above
+    // its own; it is kept iff rank < k_t.  The kept tokens go, ascending, to the frame's staging row.
+    unsigned long long* comp = reinterpret_cast<unsigned long long*>(&g_sum[0][0]);   // the slice sums are spent
+    __syncthreads();                        // k_t is out, g_sum is free
+    const int kt = f_fl[0];
+    unsigned long long mine = ~0ull;
+    if (tid < kMaxTokensFused) {
+        if (tid < p.f) mine = ((unsigned long long)order_key(my_I) << 32) | (0xffffffffu - (uint32_t)tid);
+        comp[tid] = tid < p.f ? mine : 0ull;
+    }
+    __syncthreads();
+    int keep = 0;
+    if (tid < p.f && kt > 0) {
+        int rank = 0;
+        const int fpad = (p.f + 1) & ~1;
+        for (int j2 = 0; j2 < fpad; j2 += 2) {
+            const ulonglong2 c2 = *reinterpret_cast<const ulonglong2*>(comp + j2);
+            rank += (c2.x > mine) + (c2.y > mine);
+        }
+        keep = rank < kt;
+    }
+    int total;
+    const int pos = block_exclusive_scan<kFinThreads>(keep, reinterpret_cast<int*>(red), total);
+    if (keep) p.kept_local[(int64_t)t * p.f + pos] = tid;
+}
+
+// Second half of the single-call stage one: the kept lists of the frames become one ascending list of
+// global token indices, and the kept rows are copied (Section 3.1: the retained tokens form the pruned
+// visual sequence).  Persistent CTAs; every CTA first scans the budgets (up to kEmitInlineFrames
+// frames; beyond, a scan kernel in front has left the offsets in kept_offsets), then takes half rows
+// in a grid-stride loop: one warp per half row, 128-bit copies.
+constexpr int kEmitThreads = 256;
+constexpr int kEmitInlineFrames = 4096;
+
+__global__ void __launch_bounds__(kEmitThreads)
+emit_gather_kernel(const int32_t* __restrict__ k, const int32_t* __restrict__ kept_local, int F, int f,
+                   int offsets_ready, int32_t* __restrict__ kept_offsets, int32_t* __restrict__ num_kept,
+                   int32_t* __restrict__ out_kept_index, int64_t capacity, const char* __restrict__ src,
+                   int64_t src_row_bytes, int nvec, char* __restrict__ dst, int64_t dst_row_bytes,
+                   int32_t* status_word) {
+    __shared__ int32_t off_s[kEmitInlineFrames + 1];
+    __shared__ int scan_sm[kEmitThreads / 32 + 1];
+    const int tid = threadIdx.x, lane = tid & 31;
+    cudaGridDependencySynchronize();        // budgets and kept lists come from the kernel in front
+    int64_t n_total;
+    if (!offsets_ready) {
+        // exclusive scan of the clamped budgets: thread i owns a contiguous share
+        const int per = (F + kEmitThreads - 1) / kEmitThreads;
+        const int lo = min(F, tid * per), hi = min(F, lo + per);
+        int sum = 0;
+        for (int i = lo; i < hi; ++i) sum += min(max(k[i], 0), f);
+        int total;
+        int run = block_exclusive_scan<kEmitThreads>(sum, scan_sm, total);
+        for (int i = lo; i < hi; ++i) {
+            off_s[i] = run;
+            run += min(max(k[i], 0), f);
+        }
+        if (tid == 0) off_s[F] = total;
+        __syncthreads();
+        n_total = total;
+        if (blockIdx.x == 0) {
+            for (int i = tid; i <= F; i += kEmitThreads) kept_offsets[i] = off_s[i];
+            if (tid == 0) {
+                if (num_kept) *num_kept = total;
+                if ((int64_t)total > capacity) report(status_word, SHARPV_ERR_CAPACITY);
+            }
+        }
+    } else {
+        n_total = kept_offsets[F];
+    }
+    const int64_t n = min(n_total, capacity);
+    const int half = (nvec + 1) >> 1;
+    for (int64_t w = (int64_t)blockIdx.x * (kEmitThreads / 32) + (tid >> 5); w < 2 * n;
+         w += (int64_t)gridDim.x * (kEmitThreads / 32)) {
+        const int64_t j = w >> 1;
+        const int t = offsets_ready ? upper_segment(kept_offsets, F, (int)j) : upper_segment_any(off_s, F, (int)j);
+        const int base = offsets_ready ? __ldg(kept_offsets + t) : off_s[t];
+        const int32_t row_index = t * f + __ldg(kept_local + (int64_t)t * f + (j - base));
+        if ((w & 1) == 0 && lane == 0) out_kept_index[j] = row_index;
+        if (!dst) continue;
+        const int v0 = (int)(w & 1) * half, v1 = min(nvec, v0 + half);
+        const char* s = src + (int64_t)row_index * src_row_bytes;
+        char* o = dst + j * dst_row_bytes;
+        for (int v = v0 + lane; v < v1; v += 256) {
+            uint4 r[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (v + 32 * u < v1) r[u] = ld_stream(s + (int64_t)(v + 32 * u) * 16);
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (v + 32 * u < v1) st_stream(o + (int64_t)(v + 32 * u) * 16, r[u]);
+        }
     }
 }
 
@@ -515,6 +615,28 @@ sharpv_status launch(const FusedScoreArgs& a, FusedParams& p, int dev, int sms) 
         (void)cudaGetLastError();
         return SHARPV_ERR_CUDA;
     }
+    if (!a.select) return SHARPV_OK;
+
+    // single-call stage one: offsets of the frames' kept lists, one global list, the kept rows
+    const int offsets_ready = a.F > kEmitInlineFrames;
+    if (offsets_ready &&
+        launch_dependent(exclusive_scan_i32_kernel<true>, dim3(1), dim3(kScanThreads), 0, a.stream,
+                         (const int32_t*)a.out_k, (int64_t)a.F, (int)a.f, a.out_kept_offsets, a.out_kept_offsets + a.F,
+                         a.out_num_kept, a.capacity, a.status_word) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SHARPV_ERR_CUDA;
+    }
+    const int64_t rows = a.capacity < (int64_t)a.F * a.f ? a.capacity : (int64_t)a.F * a.f;
+    const int64_t want = (2 * rows + kEmitThreads / 32 - 1) / (kEmitThreads / 32);
+    const int64_t most = (int64_t)sms * 8;
+    const unsigned egrid = (unsigned)(want < 1 ? 1 : (want < most ? want : most));
+    if (launch_dependent(emit_gather_kernel, dim3(egrid), dim3(kEmitThreads), 0, a.stream, (const int32_t*)a.out_k,
+                         (const int32_t*)p.kept_local, (int)a.F, (int)a.f, offsets_ready, a.out_kept_offsets,
+                         a.out_num_kept, a.out_kept_index, a.capacity, (const char*)a.tokens, p.row_bytes_ld, p.nvec,
+                         (char*)a.out_tokens, (int64_t)a.d * elem_bytes(a.dtype), a.status_word) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return SHARPV_ERR_CUDA;
+    }
     return SHARPV_OK;
 }
 
@@ -545,6 +667,8 @@ size_t fused_score_workspace_bytes(int F, int f, int d) {
     return align_up((size_t)F * d * 4, 256) + align_up((size_t)F * nsl_max * f * 16, 256);
 }
 
+size_t fused_select_workspace_bytes(int F, int f) { return align_up((size_t)F * f * 4, 256); }
+
 sharpv_status fused_score_launch(const FusedScoreArgs& a) {
     const int eb = elem_bytes(a.dtype);
     FusedParams p;
@@ -560,6 +684,8 @@ sharpv_status fused_score_launch(const FusedScoreArgs& a) {
     char* w = (char*)a.workspace;
     p.mean = (float*)w;       w += align_up((size_t)a.F * a.d * 4, 256);
     p.part = (float4*)w;
+    // the staging rows of the kept lists sit behind the largest extent the scores' scratch can have
+    p.kept_local = a.select ? (int32_t*)((char*)a.workspace + fused_score_workspace_bytes(a.F, a.f, a.d)) : nullptr;
 
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||

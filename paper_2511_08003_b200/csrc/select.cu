@@ -21,12 +21,6 @@ constexpr int kMaxTokensPerFrame = 8192;
 constexpr int kRankMaxTokens = 1024;     // frames up to this size are selected by counting ranks
 constexpr int kInlineOffsetFrames = 4096; // up to this many frames every frame CTA adds up the budgets in front of it itself
 
-// Monotone map fp32 -> uint32: larger score, larger key.  Adding +0 turns -0 into +0.
-__device__ __forceinline__ uint32_t order_key(float x) {
-    const uint32_t b = __float_as_uint(x + 0.0f);
-    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
-
 __global__ void __launch_bounds__(kSelectThreads)
 count_above_kernel(const float* __restrict__ importance, float K, int f, int32_t* __restrict__ counts) {
     __shared__ int part[kSelectThreads / 32];

@@ -78,6 +78,33 @@ def test_score_frames_rejects_bad_arguments(L):
     assert call(F=0) == S.OK                            # empty input: nothing launched
 
 
+def test_prune_frames_rejects_bad_arguments(L):
+    ok = dict(tokens=P, dtype=1, ld=3584, nv=1, vfo=P, F=4, f=196, d=3584, w=1.0, kind=0, rm=0, mk=0,
+              I=P, S=None, T=None, r=P, k=P, ki=P, ko=P, ot=P, cap=784, nk=P, ws=P, wsb=1 << 30, st=None, stream=None)
+
+    def call(**kw):
+        a = dict(ok, **kw)
+        return L.sharpv_prune_frames(a["tokens"], a["dtype"], a["ld"], a["nv"], a["vfo"], a["F"], a["f"], a["d"],
+                                     a["w"], a["kind"], a["rm"], a["mk"], a["I"], a["S"], a["T"], a["r"], a["k"],
+                                     a["ki"], a["ko"], a["ot"], a["cap"], a["nk"], a["ws"], a["wsb"], a["st"],
+                                     a["stream"])
+
+    S = sv.Status
+    assert L.sharpv_prune_frames_workspace_bytes(32, 196, 3584) >= (
+        L.sharpv_score_frames_workspace_bytes(32, 196, 3584))
+    assert call(dtype=2) == S.ERR_UNSUPPORTED
+    assert call(tokens=None) == S.ERR_INVALID_ARG
+    assert call(ko=None) == S.ERR_INVALID_ARG
+    assert call(ki=None) == S.ERR_INVALID_ARG
+    assert call(cap=-1) == S.ERR_INVALID_ARG
+    assert call(f=0) == S.ERR_INVALID_ARG
+    assert call(ld=100) == S.ERR_INVALID_ARG
+    assert call(kind=2) == S.ERR_INVALID_ARG
+    assert call(d=3, ld=3) == S.ERR_UNSUPPORTED
+    assert call(ot=P + 4) == S.ERR_UNSUPPORTED
+    assert call(wsb=1024) == S.ERR_WORKSPACE
+
+
 def test_select_tokens_rejects_bad_arguments(L):
     def call(imp=P, k=P, F=4, f=196, tok=P, dt=1, ld=3584, d=3584, idx=P, off=P, out=P, cap=100, nk=None, ws=P,
              wsb=1 << 20, st=None):
