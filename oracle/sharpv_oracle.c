@@ -283,6 +283,70 @@ int64_t sharpv_oracle_kv_calibrate_prune(const void *hidden, int64_t ld_hidden,
 }
 
 /*
+ * Stage two read as Eq. 7 is printed (Section 3.2.3): Discard = cos(V_l, V) < M is one decision per
+ * layer l, taken on the similarity between the layer's visual hidden states V_l and the original
+ * visual features V; the similarity of two token matrices is the average of the token-wise cosines
+ * (the per-layer average similarity of Section 3.2.1, Fig. 3), taken per sequence.  A layer that
+ * fails the test loses the K/V of its visual tokens, and so does every deeper layer ("hierarchical"
+ * pruning, Section 1; Section 4.3.2 counts the layers below the threshold); text tokens are never
+ * dropped.
+ *   hidden: n_layers hidden states, layer i at hidden + i * stride_layer elements, each [T, d];
+ *   mean_cos [n_layers * B]: average cosine of sequence b at layer i (0 for a sequence without
+ *     visual tokens);
+ *   first_discard [B]: the first layer index i with mean_cos < M (decided in fp32), n_layers if none;
+ *   per layer i: kept_pos + i * T (ascending packed positions) and kept_seq_offsets + i * (B + 1).
+ * Returns 0 or -1.
+ */
+int sharpv_oracle_kv_discard_layers(const void *hidden, int64_t stride_layer, int64_t ld_hidden,
+                                    const void *visual, int64_t ld_visual, int dtype, int d,
+                                    int n_layers, int num_seqs, const int32_t *seq_offsets,
+                                    const int32_t *vis_begin, const int32_t *vis_count,
+                                    const int32_t *vis_offsets, double M,
+                                    double *mean_cos, int32_t *first_discard,
+                                    int32_t *kept_pos, int32_t *kept_seq_offsets, int nthreads)
+{
+    if (!hidden || !visual || !seq_offsets || num_seqs < 1 || d < 1 || n_layers < 0) return -1;
+    if (nthreads < 1) nthreads = 1;
+    int64_t T = seq_offsets[num_seqs];
+    int fail = 0;
+    for (int b = 0; b < num_seqs; ++b) first_discard[b] = n_layers;
+    for (int i = 0; i < n_layers; ++i) {
+        for (int b = 0; b < num_seqs; ++b) {
+            int64_t base = (int64_t)seq_offsets[b] + vis_begin[b];
+            double sum = 0.0;
+#pragma omp parallel for num_threads(nthreads) schedule(static) reduction(+ : sum)
+            for (int r = 0; r < vis_count[b]; ++r) {
+                double *h = (double *)malloc(sizeof(double) * (size_t)d);
+                double *v = (double *)malloc(sizeof(double) * (size_t)d);
+                if (!h || !v) { fail = 1; free(h); free(v); continue; }
+                /* layer i starts stride_layer elements further on */
+                for (int j = 0; j < d; ++j)
+                    h[j] = load_elem(hidden, dtype, (int64_t)i * stride_layer + (base + r) * ld_hidden + j);
+                load_row(visual, dtype, (int64_t)vis_offsets[b] + r, ld_visual, d, v);
+                sum += sharpv_oracle_cosine(h, v, d);
+                free(h); free(v);
+            }
+            double mean = vis_count[b] > 0 ? sum / (double)vis_count[b] : 0.0;
+            mean_cos[(int64_t)i * num_seqs + b] = mean;
+            if (vis_count[b] > 0 && first_discard[b] == n_layers && (float)mean < (float)M)
+                first_discard[b] = i;                       /* Eq. 7, and every deeper layer with it */
+        }
+        int32_t *kp = kept_pos + (int64_t)i * T;
+        int32_t *kso = kept_seq_offsets + (int64_t)i * (num_seqs + 1);
+        int64_t n = 0;
+        for (int b = 0; b < num_seqs; ++b) {
+            kso[b] = (int32_t)n;
+            int dropped = i >= first_discard[b];
+            int64_t v0 = (int64_t)seq_offsets[b] + vis_begin[b], v1 = v0 + vis_count[b];
+            for (int64_t p = seq_offsets[b]; p < seq_offsets[b + 1]; ++p)
+                if (!(dropped && p >= v0 && p < v1)) kp[n++] = (int32_t)p;
+        }
+        kso[num_seqs] = (int32_t)n;
+    }
+    return fail ? -1 : 0;
+}
+
+/*
  * Stage two, K/V compaction: for every layer in [layer_begin, layer_end), K and V,
  * and KV head, dst[j, :] = src[kept_pos[j], :] for j < n_kept.  Strides in bytes;
  * the head_dim axis is contiguous (row_bytes bytes).

@@ -218,6 +218,38 @@ def kv_prune_layers(hidden_layers, visual: np.ndarray, seq_offsets, vis_begin, v
     return results, out
 
 
+def kv_discard_layers(hidden_layers: np.ndarray, visual: np.ndarray, seq_offsets, vis_begin, vis_count,
+                      vis_offsets, M: float, nthreads: int = 1):
+    """Eq. 7 as printed: one decision per layer (and sequence) on the average cosine between the layer's
+    visual hidden states and the original features; the first failing layer and every deeper one lose
+    their visual K/V rows.  hidden_layers: [n_layers, T, d].  Returns dict(mean_cos [n, B] f64,
+    first_discard [B] int32 (n if none), kept_pos: list of n ascending int32 arrays,
+    kept_seq_offsets [n, B+1])."""
+    assert hidden_layers.ndim == 3 and hidden_layers.strides[2] == hidden_layers.itemsize
+    so = np.ascontiguousarray(seq_offsets, dtype=np.int32)
+    vb = np.ascontiguousarray(vis_begin, dtype=np.int32)
+    vc = np.ascontiguousarray(vis_count, dtype=np.int32)
+    vo = np.ascontiguousarray(vis_offsets, dtype=np.int32)
+    n, T, d = hidden_layers.shape
+    B = so.size - 1
+    assert T == int(so[-1])
+    it = hidden_layers.itemsize
+    mean = np.zeros((n, B), np.float64)
+    first = np.zeros(B, np.int32)
+    kept = np.zeros((max(n, 1), max(T, 1)), np.int32)
+    kso = np.zeros((max(n, 1), B + 1), np.int32)
+    fn = lib().sharpv_oracle_kv_discard_layers
+    fn.restype = C.c_int
+    rc = fn(_ptr(hidden_layers), C.c_int64(hidden_layers.strides[0] // it), C.c_int64(hidden_layers.strides[1] // it),
+            _ptr(visual), C.c_int64(_row_major(visual)), C.c_int(_dtype_code(visual)), C.c_int(d), C.c_int(n),
+            C.c_int(B), _ptr(so), _ptr(vb), _ptr(vc), _ptr(vo), C.c_double(M), _ptr(mean), _ptr(first), _ptr(kept),
+            _ptr(kso), C.c_int(nthreads))
+    if rc != 0:
+        raise RuntimeError("sharpv_oracle_kv_discard_layers failed")
+    return dict(mean_cos=mean, first_discard=first, kept_pos=[kept[i, :kso[i, -1]].copy() for i in range(n)],
+                kept_seq_offsets=kso[:n])
+
+
 def kv_compact_rope(kv_src: np.ndarray, kept_pos, kept_seq_offsets, seq_offsets, rotary_dim: int, base: float,
                     layer_begin: int = 0, layer_end: Optional[int] = None) -> np.ndarray:
     """Compaction with rotary re-encoding of the keys.  Returns float64 [L', 2, H, n_kept, D_h]."""

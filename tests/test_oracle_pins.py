@@ -470,6 +470,58 @@ def test_layer_by_layer_pruning_is_eq7_per_layer_in_numpy():
     assert len(set(sizes)) > 1                                      # the layers really differ
 
 
+def test_layer_level_discard_is_eq7_on_the_layer_average_in_numpy():
+    """Eq. 7 as printed, against numpy on a stack of hidden states whose similarity to the visual features
+    decays with depth: per-layer average cosine, the first layer under M, and "that layer and every deeper
+    one lose their visual rows, text rows stay" (Section 3.2.3, Section 1)."""
+    rng = np.random.default_rng(31)
+    d, n_layers = 48, 7
+    lens_sys, lens_vis, lens_txt = [2, 0, 1], [11, 6, 0], [3, 2, 4]
+    so = np.concatenate([[0], np.cumsum(np.add(np.add(lens_sys, lens_vis), lens_txt))]).astype(np.int32)
+    vb = np.array(lens_sys, np.int32)
+    vc = np.array(lens_vis, np.int32)
+    vo = np.concatenate([[0], np.cumsum(lens_vis)])[:-1].astype(np.int32)
+    T = int(so[-1])
+    vis = rng.standard_normal((int(vc.sum()), d)).astype(np.float32)
+    # the second sequence drifts three times as fast as the first: it crosses the threshold earlier
+    drift = {0: [0.1, 0.3, 0.5, 0.9, 1.4, 0.6, 3.0], 1: [0.3, 0.9, 1.5, 2.7, 4.2, 1.8, 9.0]}
+    hid = rng.standard_normal((n_layers, T, d)).astype(np.float32)
+    for l in range(n_layers):
+        for b in (0, 1):
+            r0 = so[b] + vb[b]
+            hid[l, r0:r0 + vc[b]] = vis[vo[b]:vo[b] + vc[b]] + drift[b][l] * rng.standard_normal((vc[b], d))
+    M = 0.6
+    o = orc.kv_discard_layers(hid, vis, so, vb, vc, vo, M)
+    # numpy, written independently
+    mean = np.zeros((n_layers, 3))
+    for l in range(n_layers):
+        for b in (0, 1):
+            h = hid[l, so[b] + vb[b]:so[b] + vb[b] + vc[b]].astype(np.float64)
+            v = vis[vo[b]:vo[b] + vc[b]].astype(np.float64)
+            mean[l, b] = np.mean(np.sum(h * v, 1) / (np.linalg.norm(h, axis=1) * np.linalg.norm(v, axis=1)))
+    np.testing.assert_allclose(o["mean_cos"], mean, atol=1e-12)
+    first = [int(np.argmax(mean[:, b] < M)) if (mean[:, b] < M).any() else n_layers for b in (0, 1)] + [n_layers]
+    assert list(o["first_discard"]) == first
+    assert 0 < first[1] < first[0] < n_layers              # the faster drift is cut earlier; both are cut somewhere
+    # layer 5 of sequence 0 drifts less than layer 4: a layer behind the first failing one stays dropped
+    assert mean[5, 0] > mean[4, 0]
+    for l in range(n_layers):
+        want = [p for b in range(3) for p in range(so[b], so[b + 1])
+                if not (l >= first[b] and so[b] + vb[b] <= p < so[b] + vb[b] + vc[b])]
+        assert list(o["kept_pos"][l]) == want
+        assert list(o["kept_seq_offsets"][l]) == [int(np.searchsorted(want, so[b])) for b in range(4)]
+    # M below every average keeps everything at every layer; M above every average drops all visual rows at layer 0
+    lo = orc.kv_discard_layers(hid, vis, so, vb, vc, vo, -1.0)
+    assert all(k.size == T for k in lo["kept_pos"]) and list(lo["first_discard"]) == [n_layers] * 3
+    hi = orc.kv_discard_layers(hid, vis, so, vb, vc, vo, 1.5)
+    assert list(hi["first_discard"]) == [0, 0, n_layers]    # the sequence without visual tokens is never cut
+    assert all(k.size == T - int(vc.sum()) for k in hi["kept_pos"])
+    # thread count does not change anything but rounding order of the mean
+    o4 = orc.kv_discard_layers(hid, vis, so, vb, vc, vo, M, nthreads=4)
+    np.testing.assert_allclose(o4["mean_cos"], o["mean_cos"], atol=1e-14)
+    assert list(o4["first_discard"]) == first
+
+
 def test_kv_compact_inplace_equals_out_of_place_prefix():
     rng = np.random.default_rng(35)
     L, H, T, Dh = 2, 3, 41, 8
