@@ -63,7 +63,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-workload", action="store_true",
                     help="skip the per-kernel timings of the other configurations")
-    ap.add_argument("--stage", default=None, choices=list(STAGES),
+    ap.add_argument("--stage", default=None, choices=list(STAGES) + ["layers"],
                     help="profiling aid: after the warm-up run only this entry point --steps times "
                          "(HBM-cold inputs) and print its duration")
     ap.add_argument("--inplace", action="store_true",
@@ -484,6 +484,36 @@ def run_sharpv(args):
     W_ = max(args.warmup, 3)
     path.warm(W_)
     n_keep, t_keep = path.n_keep, path.t_keep
+
+    if args.stage == "layers":
+        # Stage two layer by layer over all K/V layers of the workload, both readings (profiling aid).  The
+        # hidden state of layer l is the visual feature plus noise that grows with depth, drawn on the device.
+        L = wl.num_layers
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(wl.seed * 1000 + 7)
+        hid = torch.empty((L, T, d), dtype=path.hidden.dtype, device=dev)
+        for l in range(L):
+            hid[l] = torch.randn((T, d), dtype=torch.float32, device=dev, generator=gen).to(hid.dtype)
+            hid[l, :NV] = (path.tokens.float() + (0.2 + 0.1 * l) * hid[l, :NV].float()).to(hid.dtype)
+        ws = torch.empty(sv.sharpv_kv_prune_layers_workspace_bytes(T, wl.num_videos, L), dtype=torch.uint8, device=dev)
+        tabs = [path.tabs[k] for k in ("seq_offsets", "vis_begin", "vis_count", "vis_offsets")]
+        res = {}
+        for name, mode in (("per_token", sv.PRUNE_PER_TOKEN), ("per_layer", sv.PRUNE_PER_LAYER)):
+            def call(i=0, mode=mode):
+                return sv.sharpv_kv_prune_layers(hid, path.tokens, *tabs, T, path.kv, path.kv_dst, M=args.M, mode=mode,
+                                                 workspace=ws, status_word=path.status)
+            out = call()
+            torch.cuda.synchronize()
+            kept = out["kept_seq_offsets"][:, -1].long()
+            path.stages["layers"] = call
+            tm = path.time_stage("layers", replays=max(3, min(args.steps, KERNEL_REPLAYS)), inner=1)
+            planes_row = 2 * wl.num_kv_heads * wl.head_dim * wl.elem_bytes
+            nbytes = int(L * 2 * NV * d * wl.elem_bytes + 2 * planes_row * int(kept.sum().item()))
+            res[name] = {"ms": round(tm["median_ms"], 5), "best_ms": round(tm["best_ms"], 5),
+                         "algorithmic_bytes": nbytes, "GBps": round(nbytes / (tm["median_ms"] * 1e-3) / 1e9, 1),
+                         "kept_first_layer": int(kept[0].item()), "kept_last_layer": int(kept[-1].item())}
+        print(json.dumps({"stage": "layers", "workload": args.workload, "layers": L, "M": args.M, **res}))
+        return
 
     if args.stage:
         t = path.time_stage(args.stage, replays=max(3, min(args.steps, KERNEL_REPLAYS)),

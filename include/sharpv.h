@@ -48,7 +48,9 @@ typedef enum {
     SHARPV_ERR_WORKSPACE = 3,     /* workspace smaller than the matching *_workspace_bytes() */
     SHARPV_ERR_CAPACITY = 4,      /* (status_word only) more survivors than `capacity` */
     SHARPV_ERR_CUDA = 5,          /* a CUDA runtime call or launch failed */
-    SHARPV_ERR_TIMEOUT = 6        /* (status_word only) reserved: a bounded device-side wait gave up; no kernel waits that way at present */
+    SHARPV_ERR_TIMEOUT = 6,       /* (status_word only) reserved: a bounded device-side wait gave up; no kernel waits that way at present */
+    SHARPV_ERR_BOUNDS = 7         /* (status_word only, libraries built with -DSHARPV_DEBUG_BOUNDS) an index that a kernel was
+                                     about to gather from or scatter to lay outside its range; the access was skipped */
 } sharpv_status;
 
 /* SHARPV_U8 (any one-byte element, e.g. an fp8 K/V cache) is accepted by sharpv_kv_compact only: rows are
@@ -265,10 +267,18 @@ sharpv_status sharpv_kv_compact(
 /* ------------------------------------------------------------------------------------------
  * Stage two read layer by layer.  Section 3.2.3 states Eq. 7 on the hidden state of a layer l and drops
  * "the corresponding layer's" K/V; Table 1 lists the method as adaptive per layer and Section 1 calls the
- * result a hierarchical cache pruning.  This entry point applies sharpv_kv_calibrate_prune and
- * sharpv_kv_compact once per layer l in [layer_begin, layer_end): layer l is calibrated on its own
- * hidden state and only its own K and V planes are compacted with its own kept list, so deeper layers
- * may keep fewer tokens than shallow ones.
+ * result a hierarchical cache pruning.  All layers l in [layer_begin, layer_end) are handled by the same
+ * few launches, whatever their number.  Two readings:
+ *
+ * SHARPV_PRUNE_PER_TOKEN  sharpv_kv_calibrate_prune on every layer's own hidden state and
+ *   sharpv_kv_compact of only that layer's K and V planes with that layer's kept list, so deeper layers
+ *   may keep fewer tokens than shallow ones.
+ * SHARPV_PRUNE_PER_LAYER  Eq. 7 as it is printed, Discard = cos(V_l, V) < M: one decision per layer (and
+ *   sequence) on the average, over the sequence's visual tokens, of the cosine between the layer's
+ *   hidden state and the original feature (the per-layer similarity of Section 3.2.1).  The first layer
+ *   whose average is under M loses the K/V rows of all visual tokens of that sequence, and so does
+ *   every deeper layer of the range; system and instruction tokens are never dropped; a sequence
+ *   without visual tokens is never cut.  The decision is taken on the device: no host synchronisation.
  *
  * hidden [dev]: the hidden states of the layers in the range, layer l at
  *   hidden + (l - layer_begin) * stride_hidden_layer elements, each [total_seq_tokens, d] with row
@@ -276,18 +286,25 @@ sharpv_status sharpv_kv_compact(
  * Outputs are per layer, layer l at index i = l - layer_begin:
  *   out_cos [dev] float[i * total_visual ...], out_mean_cos [dev] float[i * num_seqs ...] or NULL,
  *   out_kept_pos [dev] int32[i * capacity ...], out_kept_seq_offsets [dev] int32[i * (num_seqs + 1) ...].
- * kv_src / kv_dst and their layouts as in sharpv_kv_compact (kv_dst == kv_src compacts in place); rows of
- * a layer's planes at and beyond that layer's kept count are left untouched.  All other arguments, the
- * workspace (sharpv_kv_calibrate_prune_workspace_bytes, shared by the layers, which run one after the
- * other on the stream) and the error behaviour are those of the two entry points it is made of.
+ *   out_first_discard [dev] int32[num_seqs] or NULL (per-layer reading only; must be NULL otherwise): the
+ *   first discarded layer of each sequence, layer_end if none.
+ * kv_src / kv_dst and their layouts as in sharpv_kv_compact (kv_dst == kv_src compacts in place; both NULL:
+ * decisions only, no compaction); rows of a layer's planes at and beyond that layer's kept count are left
+ * untouched.  Workspace: sharpv_kv_prune_layers_workspace_bytes(total_seq_tokens, num_seqs, layer_end -
+ * layer_begin) bytes.  All other arguments and the error behaviour are those of the two entry points it is
+ * made of.
  */
+typedef enum { SHARPV_PRUNE_PER_TOKEN = 0, SHARPV_PRUNE_PER_LAYER = 1 } sharpv_prune_mode;
+
+size_t sharpv_kv_prune_layers_workspace_bytes(int64_t total_seq_tokens, int32_t num_seqs, int32_t num_layers);
+
 sharpv_status sharpv_kv_prune_layers(
     const void* hidden, int64_t stride_hidden_layer, int64_t ld_hidden, const void* visual, int64_t ld_visual,
     sharpv_dtype dtype, int32_t d,
     int32_t num_seqs, const int32_t* seq_offsets, const int32_t* vis_begin,
     const int32_t* vis_count, const int32_t* vis_offsets,
-    int64_t total_seq_tokens, int64_t total_visual, float M,
-    float* out_cos, float* out_mean_cos,
+    int64_t total_seq_tokens, int64_t total_visual, float M, sharpv_prune_mode mode,
+    float* out_cos, float* out_mean_cos, int32_t* out_first_discard,
     int32_t* out_kept_pos, int32_t* out_kept_seq_offsets, int64_t capacity,
     const void* kv_src, const sharpv_kv_layout* src_layout /* [host] */,
     void* kv_dst, const sharpv_kv_layout* dst_layout /* [host] */,

@@ -26,11 +26,13 @@ class Status(enum.IntEnum):
     ERR_CAPACITY = 4
     ERR_CUDA = 5
     ERR_TIMEOUT = 6
+    ERR_BOUNDS = 7
 
 
 F32, BF16, U8 = 0, 1, 2
 ROUND_FLOOR, ROUND_NEAREST, ROUND_CEIL = 0, 1, 2
 DISSIM, ONE_MINUS_COS = 0, 1
+PRUNE_PER_TOKEN, PRUNE_PER_LAYER = 0, 1
 
 
 class SharpVError(RuntimeError):
@@ -56,7 +58,7 @@ EXPORTS = (
     "sharpv_prune_frames_workspace_bytes", "sharpv_prune_frames",
     "sharpv_kv_calibrate_prune_workspace_bytes", "sharpv_kv_calibrate_prune",
     "sharpv_kv_calibrate_prune_noalloc",
-    "sharpv_kv_prune_layers", "sharpv_kv_compact",
+    "sharpv_kv_prune_layers_workspace_bytes", "sharpv_kv_prune_layers", "sharpv_kv_compact",
     "sharpv_kv_compact_rope_workspace_bytes", "sharpv_kv_compact_rope",
 )
 
@@ -64,7 +66,9 @@ NOALLOC_MAX_SEQ_TOKENS = 262144
 
 
 def lib_path() -> str:
-    return _build.LIB_PATH
+    """The library to load: libsharpv.so next to this file, or the file SHARPV_LIBRARY names (used to run the
+    tests against the range-checking debug build, libsharpv_debug.so)."""
+    return os.environ.get("SHARPV_LIBRARY") or _build.LIB_PATH
 
 
 def lib():
@@ -107,9 +111,11 @@ def lib():
     L.sharpv_kv_calibrate_prune_noalloc.argtypes = [vp, i64, vp, i64, C.c_int, i32, i32, vp, vp, vp, vp, i64, i64,
                                                     f32, vp, vp, vp, vp, i64, vp, vp]
     L.sharpv_kv_prune_layers.restype = C.c_int
+    L.sharpv_kv_prune_layers_workspace_bytes.restype = sz
+    L.sharpv_kv_prune_layers_workspace_bytes.argtypes = [i64, i32, i32]
     L.sharpv_kv_prune_layers.argtypes = [vp, i64, i64, vp, i64, C.c_int, i32, i32, vp, vp, vp, vp, i64, i64, f32,
-                                         vp, vp, vp, vp, i64, vp, C.POINTER(KVLayout), vp, C.POINTER(KVLayout),
-                                         i32, i32, vp, sz, vp, vp]
+                                         C.c_int, vp, vp, vp, vp, vp, i64, vp, C.POINTER(KVLayout), vp,
+                                         C.POINTER(KVLayout), i32, i32, vp, sz, vp, vp]
     L.sharpv_kv_compact.restype = C.c_int
     L.sharpv_kv_compact.argtypes = [vp, C.POINTER(KVLayout), vp, C.POINTER(KVLayout), i32, i32, vp, vp, i32, i64,
                                     vp, vp]
@@ -405,14 +411,21 @@ def sharpv_kv_compact(kv_src: torch.Tensor, kv_dst: torch.Tensor, kept_pos: torc
     return kv_dst
 
 
+def sharpv_kv_prune_layers_workspace_bytes(total_seq_tokens: int, num_seqs: int, num_layers: int) -> int:
+    return int(lib().sharpv_kv_prune_layers_workspace_bytes(total_seq_tokens, num_seqs, num_layers))
+
+
 def sharpv_kv_prune_layers(hidden_layers: torch.Tensor, visual: torch.Tensor, seq_offsets: torch.Tensor,
                            vis_begin: torch.Tensor, vis_count: torch.Tensor, vis_offsets: torch.Tensor,
-                           total_seq_tokens: int, kv_src: torch.Tensor, kv_dst: torch.Tensor, M: float = 0.2,
-                           layer_begin: int = 0, capacity: Optional[int] = None, want_mean_cos: bool = False,
-                           workspace=None, status_word=None, stream=None):
+                           total_seq_tokens: int, kv_src: Optional[torch.Tensor], kv_dst: Optional[torch.Tensor],
+                           M: float = 0.2, mode: int = PRUNE_PER_TOKEN, layer_begin: int = 0,
+                           capacity: Optional[int] = None, want_mean_cos: bool = False, workspace=None,
+                           status_word=None, stream=None, kv_layers: Optional[int] = None):
     """Stage two layer by layer.  hidden_layers [n_layers, T, d] holds the hidden states of layers
     layer_begin .. layer_begin + n_layers - 1.  Returns dict(cos [n, total_visual], kept_pos [n, capacity],
-    kept_seq_offsets [n, B + 1][, mean_cos [n, B]]); kv_dst receives the compacted planes."""
+    kept_seq_offsets [n, B + 1][, mean_cos [n, B]][, first_discard [B] (per-layer reading)]); kv_dst
+    receives the compacted planes.  kv_src = kv_dst = None gives the decisions only (kv_layers then says
+    how many layers the model has)."""
     if hidden_layers.dim() != 3 or hidden_layers.stride(2) != 1:
         raise ValueError("hidden_layers must be [layers, tokens, d] with a contiguous last axis")
     n = hidden_layers.shape[0]
@@ -427,19 +440,28 @@ def sharpv_kv_prune_layers(hidden_layers: torch.Tensor, visual: torch.Tensor, se
     out = {"cos": torch.empty((n, max(total_visual, 1)), dtype=torch.float32, device=dev),
            "kept_pos": torch.empty((n, max(capacity, 1)), dtype=torch.int32, device=dev),
            "kept_seq_offsets": torch.empty((n, B + 1), dtype=torch.int32, device=dev)}
-    if want_mean_cos:
+    if want_mean_cos or mode == PRUNE_PER_LAYER:
         out["mean_cos"] = torch.empty((n, B), dtype=torch.float32, device=dev)
+    if mode == PRUNE_PER_LAYER:
+        out["first_discard"] = torch.empty(B, dtype=torch.int32, device=dev)
     if total_visual == 0 or capacity == 0:
         raise ValueError("sharpv_kv_prune_layers wrapper needs total_visual > 0 and capacity > 0")
-    sl, dl = kv_layout(kv_src), kv_layout(kv_dst)
-    ws = _workspace(workspace, sharpv_kv_calibrate_prune_workspace_bytes(total_seq_tokens, B), dev)
+    if (kv_src is None) != (kv_dst is None):
+        raise ValueError("kv_src and kv_dst: both or none")
+    if kv_src is not None:
+        sl, dl = kv_layout(kv_src), kv_layout(kv_dst)
+    else:
+        L = kv_layers if kv_layers is not None else layer_begin + n
+        sl = dl = KVLayout(L, 1, 16, _dtype_code(visual), 16, 16, 16, 16)
+    ws = _workspace(workspace, sharpv_kv_prune_layers_workspace_bytes(total_seq_tokens, B, n), dev)
     rc = _call("sharpv_kv_prune_layers", hidden_layers,
         _dev(hidden_layers, "hidden_layers"), hidden_layers.stride(0), hidden_layers.stride(1),
         _dev(visual, "visual"), ldv, _dtype_code(visual), visual.shape[1], B,
         _dev(seq_offsets, "seq_offsets", torch.int32), _dev(vis_begin, "vis_begin", torch.int32),
         _dev(vis_count, "vis_count", torch.int32), _dev(vis_offsets, "vis_offsets", torch.int32),
-        total_seq_tokens, total_visual, float(M), _dev(out["cos"], "cos", torch.float32),
-        _dev(out.get("mean_cos"), "mean_cos", torch.float32), _dev(out["kept_pos"], "kept_pos", torch.int32),
+        total_seq_tokens, total_visual, float(M), int(mode), _dev(out["cos"], "cos", torch.float32),
+        _dev(out.get("mean_cos"), "mean_cos", torch.float32),
+        _dev(out.get("first_discard"), "first_discard", torch.int32), _dev(out["kept_pos"], "kept_pos", torch.int32),
         _dev(out["kept_seq_offsets"], "kept_seq_offsets", torch.int32), capacity,
         _dev(kv_src, "kv_src"), C.byref(sl), _dev(kv_dst, "kv_dst"), C.byref(dl), layer_begin, layer_begin + n,
         ws.data_ptr(), ws.numel(), _dev(status_word, "status_word", torch.int32), _stream(stream))

@@ -11,6 +11,8 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libsharpv.so")
+# the same sources with -DSHARPV_DEBUG_BOUNDS: every gather / scatter index is range-checked on the device
+DEBUG_LIB_PATH = os.path.join(_PKG, "libsharpv_debug.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -30,24 +32,26 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB_PATH):
+def needs_build(path: str = LIB_PATH) -> bool:
+    if not os.path.exists(path):
         return True
-    t = os.path.getmtime(LIB_PATH)
+    t = os.path.getmtime(path)
     deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(INCLUDE, "*.h"))
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
-        return LIB_PATH
-    tmp = LIB_PATH + f".tmp{os.getpid()}"
+def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False) -> str:
+    path = DEBUG_LIB_PATH if debug_bounds else LIB_PATH
+    if not force and not needs_build(path):
+        return path
+    tmp = path + f".tmp{os.getpid()}"
     cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
+          (["-DSHARPV_DEBUG_BOUNDS"] if debug_bounds else []) + \
           ["-I", INCLUDE, "-I", CSRC, "-o", tmp] + sources()
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, path)
+    return path
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug_bounds="--debug-bounds" in sys.argv))

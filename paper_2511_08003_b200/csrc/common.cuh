@@ -33,6 +33,16 @@ inline void kv_extent(const void* base, const sharpv_kv_layout* L, int layer_beg
                       (rows - 1) * L->stride_token + L->head_dim) * eb);
 }
 
+// Rows a plane of this layout can hold if the cache is laid out without gaps: the smallest stride above
+// the token stride, in token strides.  Only the debug build's range checks use it.
+inline int64_t kv_row_limit(const sharpv_kv_layout* L) {
+    int64_t best = INT64_MAX;
+    const int64_t strides[3] = {L->stride_layer, L->stride_kv, L->stride_head};
+    for (int i = 0; i < 3; ++i)
+        if (strides[i] > L->stride_token && strides[i] / L->stride_token < best) best = strides[i] / L->stride_token;
+    return best == INT64_MAX ? ((int64_t)1 << 31) : best;
+}
+
 // true when the first `rows` rows of the planes of [layer_begin, layer_end) of two caches share bytes
 inline bool kv_ranges_overlap(const void* a, const sharpv_kv_layout* la, const void* b, const sharpv_kv_layout* lb,
                               int layer_begin, int layer_end, int64_t rows) {
@@ -185,6 +195,18 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 __device__ __forceinline__ void report(int32_t* status_word, int code) {
     if (status_word) atomicMax(status_word, code);
 }
+
+// Range check of an index right before it is used for a gather or a scatter.  In a library built with
+// -DSHARPV_DEBUG_BOUNDS a violation is recorded in the status word and the caller skips the access; in
+// the release build the check compiles away.
+#ifdef SHARPV_DEBUG_BOUNDS
+__device__ __forceinline__ bool index_ok(bool in_range, int32_t* status_word) {
+    if (!in_range) report(status_word, SHARPV_ERR_BOUNDS);
+    return in_range;
+}
+#else
+__device__ __forceinline__ bool index_ok(bool, int32_t*) { return true; }
+#endif
 
 // Exclusive prefix sums of n ints by one CTA of 1024 threads: thread i adds up a contiguous share,
 // one block scan, then every thread writes the prefixes of its share.  out[i] = sum of val(in[j]),

@@ -8,6 +8,7 @@
 // store per dense tile) were measured and lost: the copy engine's per-request cost caps 256-byte
 // rows near 2.2 TB/s of reads, against 2.7 TB/s for this kernel at the same kept share.
 #include "common.cuh"
+#include "compact.cuh"
 
 namespace sharpv {
 namespace {
@@ -20,108 +21,255 @@ struct PlaneGeom {
     int64_t src_layer, src_kv, src_head, src_token;     // bytes
     int64_t dst_layer, dst_kv, dst_head, dst_token;     // bytes
     int num_kv_heads, layer_begin, row_vecs;            // row_vecs = 16-byte vectors per row
+    int64_t row_limit;                                  // rows a source plane can hold (what a dense layout implies)
 };
 
-// Persistent CTAs walk the (plane, tile) list; a tile is kTileRows destination rows.  Each thread
-// moves kUnroll 16-byte vectors per tile, all loads issued before the first store.
-template <int kUnroll>
-__global__ void __launch_bounds__(kCompactThreads)
+// Persistent CTAs share the (plane, tile) list in contiguous runs; a tile is tile_rows destination rows.
+// Each thread moves kUnroll 16-byte vectors per tile, all loads issued before the first store.
+template <int kUnroll, bool kPerLayer>
+__global__ void __launch_bounds__(kCompactThreads, kCompactCtasPerSm)
 kv_compact_kernel(const char* __restrict__ src, char* __restrict__ dst, PlaneGeom g, int planes,
                   const int32_t* __restrict__ kept_pos, const int32_t* __restrict__ n_kept_ptr,
-                  int64_t capacity, int32_t* status_word) {
+                  int64_t kept_stride, int64_t count_stride, int64_t capacity, int32_t* status_word) {
     cudaGridDependencySynchronize();        // the index list and the cache come from earlier work on the stream
-    const int64_t n_all = __ldg(n_kept_ptr);
-    if (blockIdx.x == 0 && threadIdx.x == 0 && n_all > capacity) report(status_word, SHARPV_ERR_CAPACITY);
-    const int64_t n = min(n_all, capacity);
+    // One list for all layers (strides 0), or every layer of the range its own list and count; then the
+    // tile grid is laid out for `capacity` rows and a tile beyond its layer's count is skipped.
+    constexpr bool per_layer = kPerLayer;
+    int64_t n = capacity;
+    if (!per_layer) {
+        const int64_t n_all = __ldg(n_kept_ptr);
+        if (blockIdx.x == 0 && threadIdx.x == 0 && n_all > capacity) report(status_word, SHARPV_ERR_CAPACITY);
+        n = min(n_all, capacity);
+    }
     if (n <= 0) return;
     const int tile_rows = kCompactThreads * kUnroll / g.row_vecs;      // >= 1, checked by the host
     const int64_t tiles_per_plane = (n + tile_rows - 1) / tile_rows;
     const int64_t total_tiles = tiles_per_plane * planes;
-    for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const int plane = (int)(tile / tiles_per_plane);
-        const int64_t row0 = (tile - plane * tiles_per_plane) * tile_rows;
-        const int l = g.layer_begin + plane / (2 * g.num_kv_heads);
-        const int kv = (plane / g.num_kv_heads) & 1;
-        const int h = plane % g.num_kv_heads;
-        const char* s = src + l * g.src_layer + kv * g.src_kv + h * g.src_head;
-        char* o = dst + l * g.dst_layer + kv * g.dst_kv + h * g.dst_head;
-        const int rows = (int)min((int64_t)tile_rows, n - row0);
-        const int total = rows * g.row_vecs;
-        uint4 r[kUnroll];
-        int64_t off[kUnroll];
+    // Every CTA takes a contiguous run of tiles in (plane, row tile) order: it writes one dense stretch of
+    // a plane after the other, and where it stands (plane, layer, K|V, head, row tile) is stepped, not
+    // divided out again for every tile.
+    const int64_t t0 = blockIdx.x, t1 = total_tiles;
+    if (t0 >= t1) return;
+    // tiles are dealt out round robin; the step from one tile of this CTA to its next is a fixed number
+    // of planes and row tiles, so where the CTA stands is stepped, not divided out again
+    const int step_planes = (int)(gridDim.x / tiles_per_plane);
+    const int64_t step_rt = gridDim.x - (int64_t)step_planes * tiles_per_plane;
+    int plane = (int)(t0 / tiles_per_plane);
+    int64_t rt = t0 - (int64_t)plane * tiles_per_plane;
+    // what a thread moves in every tile: vector vv of row rr of the tile
+    int rr[kUnroll];
+    int64_t voff[kUnroll];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int q = threadIdx.x + u * kCompactThreads;
-            if (q < total) {
-                const int rr = q / g.row_vecs, vv = q - rr * g.row_vecs;
-                const int64_t j = row0 + rr;
-                r[u] = ld_stream(s + (int64_t)__ldg(kept_pos + j) * g.src_token + (int64_t)vv * 16);
-                off[u] = j * g.dst_token + (int64_t)vv * 16;
-            }
+    for (int u = 0; u < kUnroll; ++u) {
+        const int q = threadIdx.x + u * kCompactThreads;
+        rr[u] = q / g.row_vecs;
+        voff[u] = (int64_t)(q - rr[u] * g.row_vecs) * 16;
+    }
+    for (int64_t tile = t0; tile < t1; tile += gridDim.x) {
+        const int64_t row0 = rt * tile_rows;
+        const int li = plane / (2 * g.num_kv_heads), kv = (plane / g.num_kv_heads) & 1, h = plane % g.num_kv_heads;
+        const int32_t* list = per_layer ? kept_pos + li * kept_stride : kept_pos;
+        bool skip = false;
+        if (per_layer) {
+            const int64_t n_all = __ldg(n_kept_ptr + li * count_stride);
+            if (row0 == 0 && kv == 0 && h == 0 && threadIdx.x == 0 && n_all > capacity)
+                report(status_word, SHARPV_ERR_CAPACITY);
+            n = min(n_all, capacity);
+            skip = row0 >= n;
         }
+        if (!skip) {
+            const char* s = src + (g.layer_begin + li) * g.src_layer + kv * g.src_kv + h * g.src_head;
+            char* o = dst + (g.layer_begin + li) * g.dst_layer + kv * g.dst_kv + h * g.dst_head;
+            uint4 r[kUnroll];
+            int64_t off[kUnroll];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int q = threadIdx.x + u * kCompactThreads;
-            if (q < total) st_stream(o + off[u], r[u]);
+            for (int u = 0; u < kUnroll; ++u) {
+                const int64_t j = row0 + rr[u];
+                off[u] = -1;
+                if (rr[u] < tile_rows && j < n) {
+                    const int64_t from = __ldg(list + j);
+                    if (index_ok(from >= 0 && from < g.row_limit, status_word)) {
+                        r[u] = ld_stream(s + from * g.src_token + voff[u]);
+                        off[u] = j * g.dst_token + voff[u];
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+                if (off[u] >= 0) st_stream(o + off[u], r[u]);
+        }
+        plane += step_planes;
+        rt += step_rt;
+        if (rt >= tiles_per_plane) {
+            rt -= tiles_per_plane;
+            ++plane;
         }
     }
 }
 
-// In-place compaction (kv_dst == kv_src).  Row j of the result comes from row kept_pos[j] >= j, so a
-// tile of destination rows [j0, j0 + R) only reads rows at or behind j0: rows read by later tiles are
-// never overwritten by earlier ones, but a tile may overwrite rows that an earlier tile still has to
-// read.  One CTA therefore walks a plane front to back: the loads of tile k+1 are issued, a block
-// barrier orders every thread's loads of tile k before anybody's stores of tile k, then tile k is
-// stored while tile k+1 is in flight.
+// In-place compaction (kv_dst == kv_src).  Row j of the result comes from row kept_pos[j] >= j, so
+// rows are only ever moved forward, but a row may be overwritten while another row still has to be
+// read from it.  With b_0 = n (the kept count) and b_{k+1} = the first j whose source kept_pos[j] is
+// at or behind b_k, the rows j in [b_{k+1}, b_k) read sources in [b_k, b_{k-1}) (behind n for k = 0)
+// and write destinations in [b_{k+1}, b_k): inside such a level nothing that is read is written, so a
+// level is copied by all SMs at once like the out-of-place case, and the levels only have to run
+// innermost first (level k+1 reads what level k overwrites).  kInplaceLevels levels are peeled off
+// that way; the rows in front of the innermost boundary are walked front to back by one CTA per
+// plane: the loads of tile k+1 are issued, a block barrier orders every thread's loads of tile k
+// before anybody's stores of tile k, then tile k is stored while tile k+1 is in flight.  Rows that
+// stay where they are (kept_pos[j] == j) are not touched.  With a list per layer (layer-by-layer
+// call) every plane is walked front to back in full.
 constexpr int kInplaceThreads = 512;
 constexpr int kInplaceUnroll = 4;
+constexpr int kInplaceLevels = 3;
 
+// First j in [0, n) with list[j] >= x (n if there is none), list ascending.  The whole block takes
+// part (NT-ary search with __syncthreads_count); every thread returns the answer.
+// With SHIFT the searched sequence is list[j] - j (how far row j moves; non-decreasing as well).
+template <int NT, bool SHIFT = false>
+__device__ __forceinline__ int64_t block_lower_bound(const int32_t* __restrict__ list, int64_t n, int64_t x) {
+    int64_t lo = 0, hi = n;             // the answer is in [lo, hi]; list[lo - 1] < x, list[hi] >= x
+    while (hi > lo) {
+        const int64_t step = (hi - lo + NT - 1) / NT;
+        const int64_t probe = lo + (int64_t)threadIdx.x * step;
+        const int below = (probe < hi && (int64_t)__ldg(list + probe) - (SHIFT ? probe : 0) < x) ? 1 : 0;
+        const int c = __syncthreads_count(below);
+        if (c == 0) {
+            hi = lo;
+        } else {
+            const int64_t last_below = lo + (int64_t)(c - 1) * step;
+            hi = min(hi, lo + (int64_t)c * step);
+            lo = last_below + 1;
+        }
+    }
+    return lo;
+}
+
+// boundary b_{level}: b_0 = n, b_{k+1} = first j with kept_pos[j] >= b_k
+template <int NT>
+__device__ __forceinline__ void level_bounds(const int32_t* __restrict__ kept_pos, int64_t n, int level, int64_t& hi,
+                                             int64_t& lo) {
+    hi = n;
+    lo = block_lower_bound<NT>(kept_pos, hi, hi);
+    for (int k = 0; k < level; ++k) {
+        hi = lo;
+        lo = block_lower_bound<NT>(kept_pos, hi, hi);
+    }
+}
+
+// front-to-back walk of the rows [0, b_{first_level}) of every plane (first_level < 0: all n rows)
 __global__ void __launch_bounds__(kInplaceThreads)
 kv_compact_inplace_kernel(char* __restrict__ kv, PlaneGeom g, const int32_t* __restrict__ kept_pos,
-                          const int32_t* __restrict__ n_kept_ptr, int64_t capacity, int32_t* status_word) {
+                          const int32_t* __restrict__ n_kept_ptr, int64_t kept_stride, int64_t count_stride,
+                          int64_t capacity, int first_level, int32_t* status_word) {
     cudaGridDependencySynchronize();
-    const int64_t n_all = __ldg(n_kept_ptr);
-    if (blockIdx.x == 0 && threadIdx.x == 0 && n_all > capacity) report(status_word, SHARPV_ERR_CAPACITY);
-    const int64_t n = min(n_all, capacity);
-    if (n <= 0) return;
     const int plane = blockIdx.x;
-    const int l = g.layer_begin + plane / (2 * g.num_kv_heads);
+    const int li = plane / (2 * g.num_kv_heads);            // the layer's own list and count, if it has them
+    kept_pos += li * kept_stride;
+    const int64_t n_all = __ldg(n_kept_ptr + li * count_stride);
+    if (plane % (2 * g.num_kv_heads) == 0 && threadIdx.x == 0 && n_all > capacity)
+        report(status_word, SHARPV_ERR_CAPACITY);
+    int64_t n = min(n_all, capacity);
+    if (n <= 0) return;
+    if (first_level >= 0) {
+        int64_t hi, lo;
+        level_bounds<kInplaceThreads>(kept_pos, n, first_level, hi, lo);
+        n = lo;                                             // the rows behind it are copied level by level
+        if (n <= 0) return;
+    }
+    const int l = g.layer_begin + li;
     const int kvi = (plane / g.num_kv_heads) & 1;
     const int h = plane % g.num_kv_heads;
     char* base = kv + l * g.src_layer + kvi * g.src_kv + h * g.src_head;
     const int tile_rows = kInplaceThreads * kInplaceUnroll / g.row_vecs;
     const int64_t tiles = (n + tile_rows - 1) / tile_rows;
+    // the rows in front of the first one that moves stay as they are: start at its tile
+    const int64_t first_tile = block_lower_bound<kInplaceThreads, true>(kept_pos, n, 1) / tile_rows;
+    if (first_tile >= tiles) return;
 
     uint4 cur[kInplaceUnroll], nxt[kInplaceUnroll];
-    auto load_tile = [&](int64_t k, uint4 (&r)[kInplaceUnroll]) {
+    bool cur_moves[kInplaceUnroll], nxt_moves[kInplaceUnroll];
+    auto load_tile = [&](int64_t k, uint4 (&r)[kInplaceUnroll], bool (&moves)[kInplaceUnroll]) {
         const int64_t row0 = k * tile_rows;
         const int total = (int)min((int64_t)tile_rows, n - row0) * g.row_vecs;
 #pragma unroll
         for (int u = 0; u < kInplaceUnroll; ++u) {
             const int q = threadIdx.x + u * kInplaceThreads;
+            moves[u] = false;
             if (q < total) {
                 const int rr = q / g.row_vecs, vv = q - rr * g.row_vecs;
-                r[u] = *reinterpret_cast<const uint4*>(base + (int64_t)__ldg(kept_pos + row0 + rr) * g.src_token +
-                                                       (int64_t)vv * 16);
+                const int64_t from = __ldg(kept_pos + row0 + rr);
+                moves[u] = from != row0 + rr && index_ok(from > row0 + rr && from < g.row_limit, status_word);
+                if (moves[u])
+                    r[u] = *reinterpret_cast<const uint4*>(base + from * g.src_token + (int64_t)vv * 16);
             }
         }
     };
-    load_tile(0, cur);
-    for (int64_t k = 0; k < tiles; ++k) {
-        if (k + 1 < tiles) load_tile(k + 1, nxt);
+    load_tile(first_tile, cur, cur_moves);
+    for (int64_t k = first_tile; k < tiles; ++k) {
+        if (k + 1 < tiles) load_tile(k + 1, nxt, nxt_moves);
         __syncthreads();                        // every load of tile k happened before any store of tile k
         const int64_t row0 = k * tile_rows;
-        const int total = (int)min((int64_t)tile_rows, n - row0) * g.row_vecs;
 #pragma unroll
         for (int u = 0; u < kInplaceUnroll; ++u) {
             const int q = threadIdx.x + u * kInplaceThreads;
-            if (q < total) {
+            if (cur_moves[u]) {
                 const int rr = q / g.row_vecs, vv = q - rr * g.row_vecs;
                 *reinterpret_cast<uint4*>(base + (row0 + rr) * g.src_token + (int64_t)vv * 16) = cur[u];
             }
         }
 #pragma unroll
-        for (int u = 0; u < kInplaceUnroll; ++u) cur[u] = nxt[u];
+        for (int u = 0; u < kInplaceUnroll; ++u) {
+            cur[u] = nxt[u];
+            cur_moves[u] = nxt_moves[u];
+        }
+    }
+}
+
+// one level [b_{level+1}, b_level) of the in-place compaction: sources and destinations are disjoint
+// row ranges, so this is the persistent (plane, tile) walk of the out-of-place kernel on one cache
+template <int kUnroll>
+__global__ void __launch_bounds__(kCompactThreads, kCompactCtasPerSm)
+kv_compact_inplace_level_kernel(char* __restrict__ kv, PlaneGeom g, int planes, const int32_t* __restrict__ kept_pos,
+                                const int32_t* __restrict__ n_kept_ptr, int64_t capacity, int level,
+                                int32_t* status_word) {
+    cudaGridDependencySynchronize();
+    const int64_t n = min((int64_t)__ldg(n_kept_ptr), capacity);
+    if (n <= 0) return;
+    int64_t hi, lo;
+    level_bounds<kCompactThreads>(kept_pos, n, level, hi, lo);
+    const int64_t rows_all = hi - lo;
+    if (rows_all <= 0) return;
+    const int tile_rows = kCompactThreads * kUnroll / g.row_vecs;
+    const int64_t tiles_per_plane = (rows_all + tile_rows - 1) / tile_rows;
+    const int64_t total_tiles = tiles_per_plane * planes;
+    for (int64_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        const int plane = (int)(tile / tiles_per_plane);
+        const int64_t row0 = lo + (tile - plane * tiles_per_plane) * tile_rows;
+        const int l = g.layer_begin + plane / (2 * g.num_kv_heads);
+        const int kvi = (plane / g.num_kv_heads) & 1;
+        const int h = plane % g.num_kv_heads;
+        char* base = kv + l * g.src_layer + kvi * g.src_kv + h * g.src_head;
+        const int total = (int)min((int64_t)tile_rows, hi - row0) * g.row_vecs;
+        uint4 r[kUnroll];
+        int64_t off[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int q = threadIdx.x + u * kCompactThreads;
+            off[u] = -1;
+            if (q < total) {
+                const int rr = q / g.row_vecs, vv = q - rr * g.row_vecs;
+                const int64_t j = row0 + rr;
+                const int64_t from = __ldg(kept_pos + j);
+                if (from != j && index_ok(from >= hi && from < g.row_limit, status_word)) {
+                    r[u] = ld_stream(base + from * g.src_token + (int64_t)vv * 16);
+                    off[u] = j * g.src_token + (int64_t)vv * 16;
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+            if (off[u] >= 0) st_stream(base + off[u], r[u]);
     }
 }
 
@@ -141,10 +289,12 @@ bool layout_aligned(const sharpv_kv_layout* L) {
 
 using namespace sharpv;
 
-extern "C" sharpv_status sharpv_kv_compact(
-    const void* kv_src, const sharpv_kv_layout* src_layout, void* kv_dst, const sharpv_kv_layout* dst_layout,
-    int32_t layer_begin, int32_t layer_end, const int32_t* kept_pos, const int32_t* kept_seq_offsets,
-    int32_t num_seqs, int64_t capacity, int32_t* status_word, void* cuda_stream) {
+namespace sharpv {
+
+sharpv_status kv_compact_launch(const void* kv_src, const sharpv_kv_layout* src_layout, void* kv_dst,
+                                const sharpv_kv_layout* dst_layout, int32_t layer_begin, int32_t layer_end,
+                                const int32_t* kept_pos, const int32_t* n_kept_ptr, int64_t kept_stride,
+                                int64_t count_stride, int64_t capacity, int32_t* status_word, cudaStream_t stream) {
     if (!layout_ok(src_layout) || !layout_ok(dst_layout)) {
         if (src_layout && dst_layout && (!copy_dtype_ok(src_layout->dtype) || !copy_dtype_ok(dst_layout->dtype)))
             return SHARPV_ERR_UNSUPPORTED;
@@ -153,10 +303,9 @@ extern "C" sharpv_status sharpv_kv_compact(
     if (src_layout->dtype != dst_layout->dtype || src_layout->head_dim != dst_layout->head_dim ||
         src_layout->num_kv_heads != dst_layout->num_kv_heads || src_layout->num_layers != dst_layout->num_layers)
         return SHARPV_ERR_INVALID_ARG;
-    if (layer_begin < 0 || layer_end > src_layout->num_layers || layer_begin > layer_end || num_seqs < 1 ||
-        capacity < 0)
+    if (layer_begin < 0 || layer_end > src_layout->num_layers || layer_begin > layer_end || capacity < 0)
         return SHARPV_ERR_INVALID_ARG;
-    if (!kv_src || !kv_dst || !kept_seq_offsets) return SHARPV_ERR_INVALID_ARG;
+    if (!kv_src || !kv_dst || !n_kept_ptr) return SHARPV_ERR_INVALID_ARG;
     const bool in_place = kv_src == kv_dst;
     if (in_place && (src_layout->stride_layer != dst_layout->stride_layer ||
                      src_layout->stride_kv != dst_layout->stride_kv ||
@@ -186,16 +335,8 @@ extern "C" sharpv_status sharpv_kv_compact(
     g.num_kv_heads = src_layout->num_kv_heads;
     g.layer_begin = layer_begin;
     g.row_vecs = (int)(src_layout->head_dim * eb / 16);
+    g.row_limit = kv_row_limit(src_layout);
     if (g.row_vecs > kCompactThreads * kCompactUnroll) return SHARPV_ERR_UNSUPPORTED;    // rows over 16 KB
-    if (in_place) {
-        if (launch_dependent(kv_compact_inplace_kernel, dim3((unsigned)planes), dim3(kInplaceThreads), 0,
-                             (cudaStream_t)cuda_stream, (char*)kv_dst, g, kept_pos, kept_seq_offsets + num_seqs,
-                             capacity, status_word) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return SHARPV_ERR_CUDA;
-        }
-        return SHARPV_OK;
-    }
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
@@ -204,11 +345,43 @@ extern "C" sharpv_status sharpv_kv_compact(
     const int64_t max_tiles = (capacity + tile_rows - 1) / tile_rows * planes;
     const int64_t want = (int64_t)sms * kCompactCtasPerSm;
     const unsigned grid = (unsigned)(max_tiles < want ? max_tiles : want);
-    if (launch_dependent(kv_compact_kernel<kCompactUnroll>, dim3(grid), dim3(kCompactThreads), 0,
-                         (cudaStream_t)cuda_stream, (const char*)kv_src, (char*)kv_dst, g, planes, kept_pos,
-                         kept_seq_offsets + num_seqs, capacity, status_word) != cudaSuccess) {
+    if (in_place) {
+        // one list for all planes: the innermost rows front to back, then the levels, innermost first
+        const bool levels = count_stride == 0;
+        if (launch_dependent(kv_compact_inplace_kernel, dim3((unsigned)planes), dim3(kInplaceThreads), 0, stream,
+                             (char*)kv_dst, g, kept_pos, n_kept_ptr, kept_stride, count_stride, capacity,
+                             levels ? kInplaceLevels - 1 : -1, status_word) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return SHARPV_ERR_CUDA;
+        }
+        for (int level = kInplaceLevels - 1; levels && level >= 0; --level) {
+            if (launch_dependent(kv_compact_inplace_level_kernel<kCompactUnroll>, dim3(grid), dim3(kCompactThreads), 0,
+                                 stream, (char*)kv_dst, g, planes, kept_pos, n_kept_ptr, capacity, level,
+                                 status_word) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return SHARPV_ERR_CUDA;
+            }
+        }
+        return SHARPV_OK;
+    }
+    auto kern = count_stride != 0 ? kv_compact_kernel<kCompactUnroll, true> : kv_compact_kernel<kCompactUnroll, false>;
+    if (launch_dependent(kern, dim3(grid), dim3(kCompactThreads), 0, stream,
+                         (const char*)kv_src, (char*)kv_dst, g, planes, kept_pos, n_kept_ptr, kept_stride,
+                         count_stride, capacity, status_word) != cudaSuccess) {
         (void)cudaGetLastError();
         return SHARPV_ERR_CUDA;
     }
-    return launch_status();
+    return SHARPV_OK;
+}
+
+}  // namespace sharpv
+
+extern "C" sharpv_status sharpv_kv_compact(
+    const void* kv_src, const sharpv_kv_layout* src_layout, void* kv_dst, const sharpv_kv_layout* dst_layout,
+    int32_t layer_begin, int32_t layer_end, const int32_t* kept_pos, const int32_t* kept_seq_offsets,
+    int32_t num_seqs, int64_t capacity, int32_t* status_word, void* cuda_stream) {
+    if (num_seqs < 1) return SHARPV_ERR_INVALID_ARG;
+    return kv_compact_launch(kv_src, src_layout, kv_dst, dst_layout, layer_begin, layer_end, kept_pos,
+                             kept_seq_offsets ? kept_seq_offsets + num_seqs : nullptr, 0, 0, capacity, status_word,
+                             (cudaStream_t)cuda_stream);
 }

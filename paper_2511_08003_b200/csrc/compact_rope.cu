@@ -6,8 +6,13 @@
 // Values and the dimensions beyond rotary_dim are bit copies.
 //
 //   rope_table_kernel        one warp per kept row: cos / sin of its rotation angles, angles in fp64
-//   kv_compact_rope_kernel   the persistent (plane, tile) walk of the plain compaction; key vectors
-//                            inside the rotary part also fetch their partner vector and the row's
+//   kv_compact_rope_paired_kernel  (rows of a power-of-two number of vectors, at most 32) every CTA takes a
+//                            contiguous run of (row tile, plane) pairs, so the cos / sin rows of a tile
+//                            are staged in shared memory once and serve all planes; in a key plane the two
+//                            threads of a rotary pair each load their own vector, swap it with a warp
+//                            shuffle and write their own half
+//   kv_compact_rope_kernel   (other shapes) the persistent (plane, tile) walk of the plain compaction; key
+//                            vectors inside the rotary part also fetch their partner vector and the row's
 //                            cos / sin entries (L2-resident, shared by all planes)
 #include "common.cuh"
 
@@ -26,6 +31,7 @@ struct RopeGeom {
     int num_kv_heads, layer_begin, row_vecs;            // row_vecs = 16-byte vectors per row
     int rot_vecs;                                       // vectors inside the rotary part (even)
     int half;                                           // rotary_dim / 2
+    int64_t row_limit;                                  // rows a source plane can hold (debug range checks)
 };
 
 __global__ void __launch_bounds__(256)
@@ -124,8 +130,10 @@ kv_compact_rope_kernel(const char* __restrict__ src, char* __restrict__ dst, Rop
                 const int rr = q / g.row_vecs, vv = q - rr * g.row_vecs;
                 const int64_t j = row0 + rr;
                 role[u] = (kv == 0 && vv < g.rot_vecs) ? (vv < half_vecs ? 1 : 2) : 0;
+                const int64_t from = __ldg(kept_pos + j);
+                if (!index_ok(from >= 0 && from < g.row_limit, status_word)) role[u] = 2;
                 if (role[u] != 2) {
-                    const char* row = s + (int64_t)__ldg(kept_pos + j) * g.src_token + (int64_t)vv * 16;
+                    const char* row = s + from * g.src_token + (int64_t)vv * 16;
                     own[u] = ld_stream(row);
                     if (role[u] == 1) {
                         partner[u] = ld_stream(row + pair_bytes);
@@ -142,6 +150,128 @@ kv_compact_rope_kernel(const char* __restrict__ src, char* __restrict__ dst, Rop
                 st_stream(o + off[u] + pair_bytes, partner[u]);
             }
             if (role[u] != 2) st_stream(o + off[u], own[u]);
+        }
+    }
+}
+
+// Tiles in (row tile, plane) order: tile = row_tile * planes + plane.  A CTA's run of tiles stays on one
+// row tile for as long as possible, so the table rows of that tile are read from global memory once.
+template <int DT>
+__global__ void __launch_bounds__(kRopeThreads)
+kv_compact_rope_paired_kernel(const char* __restrict__ src, char* __restrict__ dst, RopeGeom g, int planes,
+                              const int32_t* __restrict__ kept_pos, const int32_t* __restrict__ n_kept_ptr,
+                              int64_t capacity, const float2* __restrict__ table, int32_t* status_word) {
+    constexpr int P = Elem<DT>::kPerVec;
+    extern __shared__ __align__(16) unsigned char rope_smem[];
+    float2* tab = reinterpret_cast<float2*>(rope_smem);        // [tile_rows][half]
+    cudaGridDependencySynchronize();
+    const int64_t n_all = __ldg(n_kept_ptr);
+    if (blockIdx.x == 0 && threadIdx.x == 0 && n_all > capacity) report(status_word, SHARPV_ERR_CAPACITY);
+    const int64_t n = min(n_all, capacity);
+    if (n <= 0) return;
+    const int tile_rows = kRopeThreads * kRopeUnroll / g.row_vecs;
+    const int64_t row_tiles = (n + tile_rows - 1) / tile_rows;
+    const int64_t total_tiles = row_tiles * planes;
+    const int64_t t0 = total_tiles * blockIdx.x / gridDim.x, t1 = total_tiles * (blockIdx.x + 1) / gridDim.x;
+    if (t0 >= t1) return;
+    const int half_vecs = g.rot_vecs >> 1;
+    int64_t staged = -1;
+    // where the run stands is stepped from tile to tile, not divided out again
+    int64_t rt = t0 / planes;
+    int plane = (int)(t0 - rt * planes);
+    int li = plane / (2 * g.num_kv_heads), kv = (plane / g.num_kv_heads) & 1, h = plane % g.num_kv_heads;
+    // what a thread handles in every tile: vector vv of row rr of the tile (rows do not straddle warps)
+    int rr[kRopeUnroll], vv[kRopeUnroll];
+#pragma unroll
+    for (int u = 0; u < kRopeUnroll; ++u) {
+        const int q = threadIdx.x + u * kRopeThreads;
+        rr[u] = q / g.row_vecs;
+        vv[u] = q - rr[u] * g.row_vecs;
+    }
+    for (int64_t tile = t0; tile < t1; ++tile) {
+        const int64_t row0 = rt * tile_rows;
+        const int rows = (int)min((int64_t)tile_rows, n - row0);
+        if (kv == 0 && g.half > 0 && staged != rt) {            // block-uniform
+            __syncthreads();                                    // nobody reads the old rows any more
+            // A thread later reads the P/2 entries (two pairs each) of its own vector, the threads of a row
+            // side by side: entry k of vector c of row r goes to (r * P/2 + k) * half_vecs + c, so that
+            // the half_vecs threads read neighbouring 16-byte words.
+            const float4* from = reinterpret_cast<const float4*>(table + row0 * g.half);
+            float4* to = reinterpret_cast<float4*>(tab);
+            const int per_row = g.half / 2;                     // 16-byte entries per row = half_vecs * P/2
+            for (int i = threadIdx.x; i < rows * per_row; i += kRopeThreads) {
+                const int r = i / per_row, m = i - r * per_row;
+                const int c = m / (P / 2), k = m - c * (P / 2);
+                to[(r * (P / 2) + k) * half_vecs + c] = __ldg(from + i);
+            }
+            __syncthreads();
+            staged = rt;
+        }
+        const char* s = src + (g.layer_begin + li) * g.src_layer + kv * g.src_kv + h * g.src_head;
+        char* o = dst + (g.layer_begin + li) * g.dst_layer + kv * g.dst_kv + h * g.dst_head;
+        uint4 own[kRopeUnroll];
+        int64_t off[kRopeUnroll];
+#pragma unroll
+        for (int u = 0; u < kRopeUnroll; ++u) {
+            own[u] = make_uint4(0u, 0u, 0u, 0u);
+            off[u] = -1;
+            if (rr[u] < rows) {
+                const int64_t j = row0 + rr[u];
+                const int64_t from = __ldg(kept_pos + j);
+                if (index_ok(from >= 0 && from < g.row_limit, status_word)) {
+                    own[u] = ld_stream(s + from * g.src_token + (int64_t)vv[u] * 16);
+                    off[u] = j * g.dst_token + (int64_t)vv[u] * 16;
+                }
+            }
+        }
+        if (kv == 0 && g.half > 0) {
+#pragma unroll
+            for (int u = 0; u < kRopeUnroll; ++u) {
+                // the partner vector of the pair sits half_vecs lanes away
+                uint4 other;
+                other.x = __shfl_xor_sync(0xffffffffu, own[u].x, half_vecs);
+                other.y = __shfl_xor_sync(0xffffffffu, own[u].y, half_vecs);
+                other.z = __shfl_xor_sync(0xffffffffu, own[u].z, half_vecs);
+                other.w = __shfl_xor_sync(0xffffffffu, own[u].w, half_vecs);
+                if (off[u] >= 0 && vv[u] < g.rot_vecs) {
+                    const bool second = vv[u] >= half_vecs;
+                    const float4* cs = reinterpret_cast<const float4*>(tab) + rr[u] * (P / 2) * half_vecs +
+                                       (vv[u] - (second ? half_vecs : 0));
+                    const float sgn = second ? 1.f : -1.f;      // x1' = x1 c - x2 s,  x2' = x2 c + x1 s
+                    float a[P], b[P], r[P];
+                    Elem<DT>::widen(own[u], a);
+                    Elem<DT>::widen(other, b);
+#pragma unroll
+                    for (int e = 0; e < P; e += 2) {
+                        const float4 t = cs[(e / 2) * half_vecs];                       // (c0, s0, c1, s1)
+                        r[e] = fmaf(a[e], t.x, b[e] * (sgn * t.y));
+                        r[e + 1] = fmaf(a[e + 1], t.z, b[e + 1] * (sgn * t.w));
+                    }
+                    if (DT == SHARPV_BF16) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const __nv_bfloat162 hh = __floats2bfloat162_rn(r[2 * e], r[2 * e + 1]);
+                            w[e] = *reinterpret_cast<const uint32_t*>(&hh);
+                        }
+                        own[u] = make_uint4(w[0], w[1], w[2], w[3]);
+                    } else {
+                        own[u] = make_uint4(__float_as_uint(r[0]), __float_as_uint(r[1]), __float_as_uint(r[P > 2 ? 2 : 0]),
+                                            __float_as_uint(r[P > 3 ? 3 : 0]));
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kRopeUnroll; ++u)
+            if (off[u] >= 0) st_stream(o + off[u], own[u]);
+        if (++plane == planes) {
+            plane = 0;
+            ++rt;
+            li = 0; kv = 0; h = 0;
+        } else if (++h == g.num_kv_heads) {
+            h = 0;
+            if (++kv == 2) { kv = 0; ++li; }
         }
     }
 }
@@ -205,6 +335,7 @@ extern "C" sharpv_status sharpv_kv_compact_rope(
     g.row_vecs = (int)(src_layout->head_dim * eb / 16);
     g.rot_vecs = (int)((int64_t)rotary_dim * eb / 16);
     g.half = rotary_dim / 2;
+    g.row_limit = kv_row_limit(src_layout);
     if (g.row_vecs > kRopeThreads * kRopeUnroll) return SHARPV_ERR_UNSUPPORTED;      // rows over 8 KB
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     float2* table = (float2*)workspace;
@@ -224,6 +355,28 @@ extern "C" sharpv_status sharpv_kv_compact_rope(
     const int64_t max_tiles = (capacity + tile_rows - 1) / tile_rows * planes;
     const int64_t want = (int64_t)sms * kRopeCtasPerSm;
     const unsigned grid = (unsigned)(max_tiles < want ? max_tiles : want);
+    // rows of a power-of-two number of vectors that fit a warp, rotary halves of a power-of-two number of
+    // vectors: the two threads of a pair sit in one warp and swap their vectors with a shuffle
+    const int half_vecs = g.rot_vecs / 2;
+    const bool pow2_row = (g.row_vecs & (g.row_vecs - 1)) == 0 && g.row_vecs <= 32;
+    const bool pow2_half = half_vecs == 0 || (half_vecs & (half_vecs - 1)) == 0;
+    const size_t tab_bytes = (size_t)tile_rows * g.half * sizeof(float2);
+    if (pow2_row && pow2_half && g.rot_vecs == 2 * half_vecs && tab_bytes <= 96 * 1024) {
+        auto kern = src_layout->dtype == SHARPV_F32 ? kv_compact_rope_paired_kernel<SHARPV_F32>
+                                                     : kv_compact_rope_paired_kernel<SHARPV_BF16>;
+        if (tab_bytes > 48 * 1024 &&
+            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tab_bytes) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return SHARPV_ERR_CUDA;
+        }
+        if (launch_dependent(kern, dim3(grid), dim3(kRopeThreads), tab_bytes, stream, (const char*)kv_src,
+                             (char*)kv_dst, g, planes, kept_pos, kept_seq_offsets + num_seqs, capacity,
+                             (const float2*)table, status_word) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return SHARPV_ERR_CUDA;
+        }
+        return SHARPV_OK;
+    }
     auto kern = src_layout->dtype == SHARPV_F32 ? kv_compact_rope_kernel<SHARPV_F32>
                                                  : kv_compact_rope_kernel<SHARPV_BF16>;
     if (launch_dependent(kern, dim3(grid), dim3(kRopeThreads), 0, stream, (const char*)kv_src, (char*)kv_dst, g,

@@ -51,6 +51,7 @@ struct FusedParams {
                             // b = the same position one frame earlier
     int32_t* kept_local;    // [F, f] or null: the finaliser also selects; frame t's kept tokens (ascending) at t * f
     int W;                  // warps per CTA: a tile is covered in R = ceil(f / 4W) visits
+    int32_t* status_word;   // may be null
 };
 
 constexpr int kBarSums = 1;     // the column sums of a tile are in shared memory
@@ -306,7 +307,7 @@ score_pass_kernel(const FusedParams p) {
             }
             float xa, xd;
             unpk(x2, xa, xd);
-            if (writes && n > 0)
+            if (writes && n > 0 && index_ok(t_prev < p.F && s_prev < p.nsl, p.status_word))
                 p.part[((int64_t)t_prev * p.nsl + s_prev) * p.f + my_row] = make_float4(keep_aa, xm, keep_db, keep_bb);
             keep_bb = keep_aa;
             keep_aa = xa;
@@ -351,7 +352,7 @@ score_pass_kernel(const FusedParams p) {
             red1_lane[4 * v * kRedStride] = hsum(bm);
         }
         __syncwarp();
-        if (writes) {
+        if (writes && index_ok(t_prev < p.F && s_prev < p.nsl, p.status_word)) {
             float xm = sum1_src[0];
 #pragma unroll
             for (int i = 1; i < 8; ++i) xm += sum1_src[i];
@@ -551,7 +552,9 @@ emit_gather_kernel(const int32_t* __restrict__ k, const int32_t* __restrict__ ke
         const int64_t j = w >> 1;
         const int t = offsets_ready ? upper_segment(kept_offsets, F, (int)j) : upper_segment_any(off_s, F, (int)j);
         const int base = offsets_ready ? __ldg(kept_offsets + t) : off_s[t];
-        const int32_t row_index = t * f + __ldg(kept_local + (int64_t)t * f + (j - base));
+        const int32_t local = __ldg(kept_local + (int64_t)t * f + (j - base));
+        if (!index_ok(j - base < f && local >= 0 && local < f, status_word)) continue;
+        const int32_t row_index = t * f + local;
         if ((w & 1) == 0 && lane == 0) out_kept_index[j] = row_index;
         if (!dst) continue;
         const int v0 = (int)(w & 1) * half, v1 = min(nvec, v0 + half);
@@ -681,6 +684,7 @@ sharpv_status fused_score_launch(const FusedScoreArgs& a) {
     p.video_frame_offsets = a.video_frame_offsets;
     p.w = a.w; p.one_minus_cos = a.one_minus_cos; p.round_mode = a.round_mode; p.min_keep = a.min_keep;
     p.out_I = a.out_I; p.out_S = a.out_S; p.out_T = a.out_T; p.out_ratio = a.out_ratio; p.out_k = a.out_k;
+    p.status_word = a.status_word;
     char* w = (char*)a.workspace;
     p.mean = (float*)w;       w += align_up((size_t)a.F * a.d * 4, 256);
     p.part = (float4*)w;

@@ -186,9 +186,9 @@ select_frame_kernel(const float* __restrict__ importance, const int32_t* __restr
 
 // one warp per half row, up to eight 128-bit loads in flight per lane
 __global__ void __launch_bounds__(256)
-gather_rows_kernel(const char* __restrict__ src, int64_t src_row_bytes, int nvec,
+gather_rows_kernel(const char* __restrict__ src, int64_t src_row_bytes, int64_t src_rows, int nvec,
                    const int32_t* __restrict__ index, const int32_t* __restrict__ count_ptr,
-                   int64_t capacity, char* __restrict__ dst, int64_t dst_row_bytes) {
+                   int64_t capacity, char* __restrict__ dst, int64_t dst_row_bytes, int32_t* status_word) {
     cudaGridDependencySynchronize();        // the index list comes from the kernel in front
     const int lane = threadIdx.x & 31;
     const int64_t w = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -198,6 +198,7 @@ gather_rows_kernel(const char* __restrict__ src, int64_t src_row_bytes, int nvec
     const int32_t row_index = __ldg(index + j);
     const int64_t n = min((int64_t)__ldg(count_ptr), capacity);
     if (j >= n) return;
+    if (!index_ok(row_index >= 0 && row_index < src_rows, status_word)) return;
     const int half = (nvec + 1) >> 1;
     const int v0 = (int)(w & 1) * half, v1 = min(nvec, v0 + half);
     const char* s = src + (int64_t)row_index * src_row_bytes;
@@ -269,9 +270,9 @@ sharpv_status select_impl(int mode, const float* importance, const int32_t* k, f
         const int64_t rows = capacity < (int64_t)F * f ? capacity : (int64_t)F * f;
         const int nvec = d * eb / 16;
         if (launch_dependent(gather_rows_kernel, dim3((unsigned)((2 * rows + 7) / 8)), dim3(256), 0, stream,
-                             (const char*)tokens, ld_tokens * eb, nvec, (const int32_t*)out_kept_index,
+                             (const char*)tokens, ld_tokens * eb, (int64_t)F * f, nvec, (const int32_t*)out_kept_index,
                              (const int32_t*)(out_kept_offsets + F), capacity, (char*)out_tokens,
-                             (int64_t)d * eb) != cudaSuccess) {
+                             (int64_t)d * eb, status_word) != cudaSuccess) {
             (void)cudaGetLastError();
             return SHARPV_ERR_CUDA;
         }

@@ -131,3 +131,28 @@ def check_kept_sets(idx_gpu, off_gpu, imp_oracle, k_used, f, select_fn, boundary
         assert np.all(np.abs(imp_oracle[sym] - kth) <= band), f"frame {t}: kept set differs away from the boundary"
         exempt += sym.size
     return exempt
+
+
+class Guarded:
+    """Device buffers with 256 bytes of a known pattern in front of and behind each of them: a kernel that
+    writes outside an output leaves a mark that check() finds (stands in for a memory checker on outputs)."""
+
+    PAD, FILL = 256, 0xA5
+
+    def __init__(self, device="cuda"):
+        self.device, self.raw = device, []
+
+    def empty(self, shape, dtype):
+        shape = (shape,) if isinstance(shape, int) else tuple(shape)
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        body = (n + 255) // 256 * 256
+        buf = torch.full((self.PAD + body + self.PAD,), self.FILL, dtype=torch.uint8, device=self.device)
+        self.raw.append((buf, n))
+        return buf[self.PAD:self.PAD + n].view(dtype).view(shape)
+
+    def check(self, what=""):
+        torch.cuda.synchronize()
+        for i, (buf, n) in enumerate(self.raw):
+            front, back = buf[:self.PAD], buf[self.PAD + n:]
+            assert bool((front == self.FILL).all()), f"{what}: bytes in front of output {i} were overwritten"
+            assert bool((back == self.FILL).all()), f"{what}: bytes behind output {i} were overwritten"

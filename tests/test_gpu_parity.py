@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import (BOUNDARY_TOL, TIGHT_TOL, TOL, DeviceWorkload, assert_scores, check_budgets, check_kept_sets, rel_err,
+from helpers import (BOUNDARY_TOL, TIGHT_TOL, TOL, DeviceWorkload, Guarded, assert_scores, check_budgets, check_kept_sets, rel_err,
                      to_dev, to_host)
 from oracle import sharpv_oracle as orc
 from paper_2511_08003_b200 import binding as sv
@@ -397,6 +397,70 @@ def test_layer_by_layer_entry_point():
         np.testing.assert_array_equal(to_host(g2["kept_seq_offsets"]), to_host(g["kept_seq_offsets"]))
     counts = [int(x) for x in to_host(g["kept_seq_offsets"])[:, -1]]
     assert counts[0] > counts[-1] >= wl.n_text          # deeper layers keep less
+
+
+def test_layer_level_discard_entry_point():
+    """Eq. 7 as printed (SHARPV_PRUNE_PER_LAYER) against the oracle: per-layer average cosine, the first
+    discarded layer of each sequence, kept lists that lose whole visual blocks from that layer on, and the
+    cache compacted with them (in place, into a second cache, decisions only); 28 layers in one call."""
+    L, lb = 30, 2
+    wl = W.custom("discard", 93, W.BF16, 6, 256, 9, [W.make_video_spec(4, 0.9), W.make_video_spec(2, 0.8),
+                                                       W.make_video_spec(3, 0.85)], 0.0, L, 2, 64)
+    W.fill_tokens(wl)
+    W.fill_kv(wl)
+    T, M, n = wl.total_seq_tokens, 0.45, L - lb
+    hidden = []
+    for i in range(n):
+        W.fill_hidden(wl, s_max=0.3 + 0.25 * i)           # the similarity decays with depth
+        hidden.append(wl.hidden.copy())
+    hid = np.stack(hidden)
+    o = orc.kv_discard_layers(hid, wl.tokens, wl.seq_offsets, wl.vis_begin, wl.vis_count, wl.vis_offsets, M, nthreads=NT)
+    first = o["first_discard"]
+    assert 0 < first.min() and first.max() < n               # every sequence is cut somewhere inside the range
+    i32 = lambda a: torch.from_numpy(a).cuda()
+    tabs = [i32(wl.seq_offsets), i32(wl.vis_begin), i32(wl.vis_count), i32(wl.vis_offsets)]
+    d_hidden = torch.from_numpy(hid.view(np.int16)).cuda().view(torch.bfloat16)
+    kv = to_dev(wl.kv)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    g = sv.sharpv_kv_prune_layers(d_hidden, to_dev(wl.tokens), *tabs, T, kv, kv, M=M, mode=sv.PRUNE_PER_LAYER,
+                                  layer_begin=lb, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    mean_g = to_host(g["mean_cos"]).astype(np.float64)
+    assert np.max(np.abs(mean_g - o["mean_cos"])) <= 1e-5
+    # a mean within 1e-5 of M may fall on either side; away from it the decisions are the oracle's
+    assert np.all(np.abs(o["mean_cos"] - M) > 1e-5), "test data sits on the threshold: change the seed"
+    np.testing.assert_array_equal(to_host(g["first_discard"]), lb + first)
+    np.testing.assert_array_equal(to_host(g["kept_seq_offsets"]), o["kept_seq_offsets"])
+    expect = wl.kv.copy()
+    for i in range(n):
+        kept = to_host(g["kept_pos"][i])[:o["kept_seq_offsets"][i, -1]]
+        np.testing.assert_array_equal(kept, o["kept_pos"][i])
+        orc.kv_compact_inplace(expect, o["kept_pos"][i], layer_begin=lb + i, layer_end=lb + i + 1)
+    np.testing.assert_array_equal(to_host(kv), expect)
+    # into a second cache; and decisions only
+    dst = torch.zeros_like(kv)
+    g2 = sv.sharpv_kv_prune_layers(d_hidden, to_dev(wl.tokens), *tabs, T, to_dev(wl.kv), dst, M=M,
+                                   mode=sv.PRUNE_PER_LAYER, layer_begin=lb)
+    g3 = sv.sharpv_kv_prune_layers(d_hidden, to_dev(wl.tokens), *tabs, T, None, None, M=M, mode=sv.PRUNE_PER_LAYER,
+                                   layer_begin=lb, kv_layers=L)
+    torch.cuda.synchronize()
+    out = to_host(dst)
+    assert np.all(out[:lb] == 0)
+    for i in range(n):
+        k = o["kept_pos"][i]
+        np.testing.assert_array_equal(out[lb + i][:, :, :k.size], wl.kv[lb + i][:, :, k])
+        assert np.all(out[lb + i][:, :, k.size:] == 0)
+    for key in ("kept_seq_offsets", "first_discard", "mean_cos"):
+        assert torch.equal(g2[key], g[key]) and torch.equal(g3[key], g[key])
+    # the per-token reading of the same stack keeps a different, token-wise set
+    g4 = sv.sharpv_kv_prune_layers(d_hidden, to_dev(wl.tokens), *tabs, T, None, None, M=M, layer_begin=lb, kv_layers=L)
+    torch.cuda.synchronize()
+    res = [orc.kv_calibrate_prune(h, wl.tokens, wl.seq_offsets, wl.vis_begin, wl.vis_count, wl.vis_offsets, M,
+                                  nthreads=NT) for h in hidden]
+    diff = sum(np.setxor1d(to_host(g4["kept_pos"][i])[:int(g4["kept_seq_offsets"][i, -1].item())],
+                           res[i]["kept_pos"]).size for i in range(n))
+    assert diff <= 4
 
 
 def test_kv_compact_one_byte_cache():
@@ -867,6 +931,74 @@ def test_many_frames_and_many_positions_use_the_scan_kernels():
     if sym.size == 0:
         np.testing.assert_array_equal(kso, o["kept_seq_offsets"])
     assert 0.2 * T < kept.size < 0.9 * T
+
+
+@pytest.mark.parametrize("name", ["tiny", "small_ragged", "odd_shapes"])
+def test_outputs_stay_inside_their_buffers(name):
+    """Every output and workspace of every entry point sits between two guard bands; capacities are exactly
+    the kept counts.  After each call the bands must be untouched."""
+    wl, dw = _case(name)
+    F, f, d, T, B = wl.total_frames, wl.f, wl.d, wl.total_seq_tokens, wl.num_videos
+    NV = F * f
+    tdt = dw.tokens.dtype
+    G = Guarded()
+    u8, f32, i32 = torch.uint8, torch.float32, torch.int32
+    # stage one, two calls
+    o1 = {"importance": G.empty(NV, f32), "spatial": G.empty(NV, f32), "temporal": G.empty(NV, f32),
+          "ratio": G.empty(F, f32), "k": G.empty(F, i32)}
+    ws1 = G.empty(sv.sharpv_score_frames_workspace_bytes(F, f, d), u8)
+    sv.sharpv_score_frames(dw.tokens, dw.video_frame_offsets, F, f, out=o1, workspace=ws1)
+    G.check("score_frames")
+    n1 = int(np.clip(to_host(o1["k"]), 0, f).sum())
+    o2 = {"kept_index": G.empty(max(n1, 1), i32), "kept_offsets": G.empty(F + 1, i32), "num_kept": G.empty(1, i32),
+          "tokens": G.empty((max(n1, 1), d), tdt)}
+    ws2 = G.empty(sv.sharpv_select_tokens_workspace_bytes(F, f), u8)
+    sv.sharpv_select_tokens(o1["importance"], o1["k"], F, f, tokens=dw.tokens, capacity=n1, out=o2, workspace=ws2)
+    G.check("select_tokens")
+    sv.sharpv_select_tokens_threshold(o1["importance"], 1.0, F, f, tokens=dw.tokens, capacity=n1, out=o2, workspace=ws2)
+    G.check("select_tokens_threshold")
+    # stage one, one call
+    o3 = {"importance": G.empty(NV, f32), "ratio": G.empty(F, f32), "k": G.empty(F, i32),
+          "kept_index": G.empty(max(n1, 1), i32), "kept_offsets": G.empty(F + 1, i32), "num_kept": G.empty(1, i32),
+          "tokens": G.empty((max(n1, 1), d), tdt)}
+    ws3 = G.empty(sv.sharpv_prune_frames_workspace_bytes(F, f, d), u8)
+    sv.sharpv_prune_frames(dw.tokens, dw.video_frame_offsets, F, f, capacity=n1, out=o3, workspace=ws3)
+    G.check("prune_frames")
+    assert int(o3["num_kept"].item()) == n1
+    # stage two
+    M = 0.6
+    tabs = (dw.seq_offsets, dw.vis_begin, dw.vis_count, dw.vis_offsets)
+    probe = sv.sharpv_kv_calibrate_prune(dw.hidden, dw.tokens, *tabs, T, M=M)
+    torch.cuda.synchronize()
+    n2 = int(probe["kept_seq_offsets"][-1].item())
+    o4 = {"cos": G.empty(NV, f32), "kept_pos": G.empty(max(n2, 1), i32), "kept_seq_offsets": G.empty(B + 1, i32),
+          "mean_cos": G.empty(B, f32)}
+    ws4 = G.empty(sv.sharpv_kv_calibrate_prune_workspace_bytes(T, B), u8)
+    sv.sharpv_kv_calibrate_prune(dw.hidden, dw.tokens, *tabs, T, M=M, capacity=n2, want_mean_cos=True, out=o4,
+                                 workspace=ws4)
+    G.check("kv_calibrate_prune")
+    sv.sharpv_kv_calibrate_prune_noalloc(dw.hidden, dw.tokens, *tabs, T, M=M, capacity=n2, want_mean_cos=True, out=o4)
+    G.check("kv_calibrate_prune_noalloc")
+    L, _, H, _, Dh = wl.kv_shape()
+    dst = G.empty((L, 2, H, max(n2, 1), Dh), tdt)
+    sv.sharpv_kv_compact(dw.kv, dst, o4["kept_pos"], o4["kept_seq_offsets"], capacity=n2)
+    G.check("kv_compact")
+    np.testing.assert_array_equal(to_host(dst)[:, :, :, :n2], wl.kv[:, :, :, to_host(o4["kept_pos"])[:n2]])
+    cache = G.empty(wl.kv_shape(), tdt)
+    cache.copy_(dw.kv)
+    sv.sharpv_kv_compact(cache, cache, o4["kept_pos"], o4["kept_seq_offsets"], capacity=n2)
+    G.check("kv_compact in place")
+    if Dh * cache.element_size() % 32 == 0:
+        wsr = G.empty(sv.sharpv_kv_compact_rope_workspace_bytes(max(n2, 1), Dh), u8)
+        sv.sharpv_kv_compact_rope(dw.kv, dst, o4["kept_pos"], o4["kept_seq_offsets"], dw.seq_offsets, n2, Dh, 1.0e4,
+                                  workspace=wsr)
+        G.check("kv_compact_rope")
+    hid = torch.stack([dw.hidden] * L)
+    wsl = G.empty(sv.sharpv_kv_prune_layers_workspace_bytes(T, B, L), u8)
+    for mode in (sv.PRUNE_PER_TOKEN, sv.PRUNE_PER_LAYER):
+        cache.copy_(dw.kv)
+        sv.sharpv_kv_prune_layers(hid, dw.tokens, *tabs, T, cache, cache, M=M, mode=mode, workspace=wsl)
+        G.check(f"kv_prune_layers mode {mode}")
 
 
 def test_run_to_run_bit_reproducible():

@@ -226,11 +226,14 @@ def test_kv_prune_layers_rejects_bad_arguments(L):
         base.update(kw)
         return sv.KVLayout(**base)
 
-    def call(hid=P, hs=500 * 512, dtype=1, sl=None, dl=None, lb=0, le=4, B=1, cap=500, ws=P, wsb=1 << 20, kso=P):
+    FAR = P + (1 << 40)
+
+    def call(hid=P, hs=500 * 512, dtype=1, sl=None, dl=None, lb=0, le=4, B=1, cap=500, ws=P, wsb=1 << 20, kso=P,
+             mode=0, fd=None):
         sl = layout() if sl is None else sl
         dl = layout() if dl is None else dl
-        return L.sharpv_kv_prune_layers(hid, hs, 512, P, 512, dtype, 512, B, P, P, P, P, 500, 400, 0.2, P, None, P, kso,
-                                        cap, P, C.byref(sl), 2 * P, C.byref(dl), lb, le, ws, wsb, None, None)
+        return L.sharpv_kv_prune_layers(hid, hs, 512, P, 512, dtype, 512, B, P, P, P, P, 500, 400, 0.2, mode, P, None,
+                                        fd, P, kso, cap, P, C.byref(sl), FAR, C.byref(dl), lb, le, ws, wsb, None, None)
 
     S = sv.Status
     assert call(lb=2, le=2) == S.OK                               # empty layer range: nothing to do
@@ -240,10 +243,13 @@ def test_kv_prune_layers_rejects_bad_arguments(L):
     assert call(hs=-1) == S.ERR_INVALID_ARG
     assert call(hs=500 * 512 + 4) == S.ERR_UNSUPPORTED            # layers of hidden states not 16-byte aligned
     assert call(B=0) == S.ERR_INVALID_ARG
-    assert call(wsb=16) == S.ERR_WORKSPACE                        # from the calibration of the first layer
+    assert call(wsb=16) == S.ERR_WORKSPACE
     assert call(kso=None) == S.ERR_INVALID_ARG
-    assert L.sharpv_kv_prune_layers(P, 0, 512, P, 512, 1, 512, 1, P, P, P, P, 500, 400, 0.2, P, None, P, P, 500, P,
-                                    None, 2 * P, None, 0, 1, P, 1 << 20, None, None) == S.ERR_INVALID_ARG
+    assert call(mode=2) == S.ERR_INVALID_ARG
+    assert call(mode=0, fd=P) == S.ERR_INVALID_ARG                # the first discarded layer exists per layer only
+    assert L.sharpv_kv_prune_layers_workspace_bytes(500, 1, 4) >= 4 * L.sharpv_kv_calibrate_prune_workspace_bytes(500, 1)
+    assert L.sharpv_kv_prune_layers(P, 0, 512, P, 512, 1, 512, 1, P, P, P, P, 500, 400, 0.2, 0, P, None, None, P, P,
+                                    500, P, None, 2 * P, None, 0, 1, P, 1 << 20, None, None) == S.ERR_INVALID_ARG
 
 
 def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
