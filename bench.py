@@ -63,6 +63,8 @@ def parse_args():
                          "(the paper's reported memory ratio); the paper's default 0.2 keeps all of them")
     ap.add_argument("--w", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-chained", action="store_true",
+                    help="skip the secondary number (stage two on the survivors of stage one)")
     ap.add_argument("--no-per-workload", action="store_true",
                     help="skip the per-kernel timings of the other configurations")
     ap.add_argument("--stage", default=None, choices=list(STAGES) + ["layers"],
@@ -76,6 +78,9 @@ def parse_args():
                     help="override the number of K/V layers (profiling aid: smaller device footprint)")
     ap.add_argument("--frames", type=int, default=None,
                     help="override the frame count of a single-video workload (profiling aid)")
+    ap.add_argument("--d", type=int, default=None,
+                    help="override the feature size (profiling aid: e.g. 3576 makes rows that are not a multiple of "
+                         "128 bytes, which take the three-kernel score path)")
     return ap.parse_args()
 
 
@@ -129,12 +134,14 @@ def oracle_step(wl, orc, M, w, nthreads, kv_layers=None):
     return t, idx.size, c["kept_pos"].size
 
 
-def host_workload(name, with_kv_layers=None, frames=None, layers=None):
+def host_workload(name, with_kv_layers=None, frames=None, layers=None, d=None):
     kw = {}
     if frames:
         kw["n_frames"] = frames
     if layers:
         kw["num_layers"] = layers
+    if d:
+        kw["d"] = d
     wl = W.PRESETS[name](**kw)
     W.fill_tokens(wl)
     W.fill_hidden(wl)
@@ -472,7 +479,7 @@ def run_sharpv(args):
     sv.lib()                                            # fail loudly before any work if not built
 
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)      # > 2x the 126 MB L2
-    wl = host_workload(args.workload, frames=args.frames, layers=args.layers)
+    wl = host_workload(args.workload, frames=args.frames, layers=args.layers, d=args.d)
     F, f, d, T, NV = wl.total_frames, wl.f, wl.d, wl.total_seq_tokens, wl.n_visual
     path = DevicePath(wl, args, dev, flush)
     stream = torch.cuda.current_stream()
@@ -574,7 +581,7 @@ def run_sharpv(args):
     # The survivors' features, hidden rows and K/V rows are laid out once with torch indexing (set-up,
     # not timed); calibration and compaction then run on that smaller sequence set.
     chained = None
-    if world == 1 and wl.num_videos == 1 and n_keep > 0 and not args.inplace and not args.rope:
+    if world == 1 and wl.num_videos == 1 and n_keep > 0 and not args.inplace and not args.rope and not args.no_chained:
         idx = path.o_sel["kept_index"][:n_keep].long()
         pos = torch.cat([idx, torch.arange(NV, T, device=dev)])            # survivors, then the text tokens
         c_vis = path.tokens.index_select(0, idx).contiguous()
@@ -655,7 +662,7 @@ def run_sharpv(args):
     dom = max(STEP_STAGES, key=lambda k: kernels[k]["median_ms"])
     cap = NCU_TRAFFIC.get((args.workload, dom))
     same_launch = (cap is not None and not args.inplace and not args.rope and args.frames is None and
-                   args.layers is None and abs(cap["M"] - args.M) < 1e-9 and cap["kept_stage_two"] == t_keep)
+                   args.layers is None and args.d is None and abs(cap["M"] - args.M) < 1e-9 and cap["kept_stage_two"] == t_keep)
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["GBps"], "peak": peak, "unit": "GB/s",
                 "frac": kernels[dom]["frac"], "peak_source": f"of {peak_kind}",
                 "frac_of_nominal_8000": kernels[dom]["frac_of_nominal_8000"],
@@ -668,7 +675,7 @@ def run_sharpv(args):
                                         ("median_ms", "best_ms", "GBps", "frac_of_measured", "frac_of_nominal_8000")}
                                     for k in STAGES}}
     per_workload[args.workload]["frames"] = F
-    if world == 1 and not args.no_per_workload and args.frames is None and args.layers is None:
+    if world == 1 and not args.no_per_workload and args.frames is None and args.layers is None and args.d is None:
         del path, graph
         torch.cuda.empty_cache()
         for name in REPORTED_WORKLOADS:
@@ -692,7 +699,7 @@ def run_sharpv(args):
         from oracle import sharpv_oracle as orc
         cores = os.cpu_count() or 1
         kv_layers = 2
-        hw = host_workload(args.workload, with_kv_layers=kv_layers, frames=args.frames)
+        hw = host_workload(args.workload, with_kv_layers=kv_layers, frames=args.frames, d=args.d)
         cpu = oracle_baseline(hw, orc, args, cores, kv_layers)
 
     cfg = workload_config(wl, args)

@@ -240,8 +240,9 @@ sharpv_status sharpv_kv_calibrate_prune_noalloc(
  * as a bit copy of head_dim elements.  Strides are in elements; the head_dim axis is
  * contiguous; every stride * sizeof(element) and head_dim * sizeof(element) must be a
  * multiple of 16 bytes; a row (head_dim elements) may be at most 16 KB.  The benchmarked layout is
- * [L][2][H][T][D_h]; a token-major cache is expressed through the strides.  kv_dst == kv_src with identical strides compacts in place (every
- * plane is walked front to back; serving stacks that cannot afford a second cache use this);
+ * [L][2][H][T][D_h]; a token-major cache is expressed through the strides.  kv_dst == kv_src with identical strides
+ * compacts in place (kept_pos must then be strictly ascending, as sharpv_kv_calibrate_prune writes it; serving
+ * stacks that cannot afford a second cache use this);
  * otherwise dst must not overlap src: the byte ranges that the first `capacity` token rows of the planes of
  * [layer_begin, layer_end) span in the two caches must be disjoint, or SHARPV_ERR_INVALID_ARG is returned and
  * nothing is launched.  Rows of dst at and beyond
@@ -319,8 +320,9 @@ sharpv_status sharpv_kv_prune_layers(
  * moves from p_old = kept_pos[j] - seq_offsets[b] to p_new = j - kept_seq_offsets[b] inside its
  * sequence b, so while its key row is copied it is rotated by (p_new - p_old):
  *     x1' = x1 cos - x2 sin,  x2' = x2 cos + x1 sin.
- * Angles are evaluated in fp64, the rotation in fp32, the result is rounded to the storage type (round
- * to nearest even).  Values and the dimensions at and beyond rotary_dim are bit copies; rotary_dim = 0
+ * Angles are formed and reduced to [-pi, pi] in fp64, their sine and cosine and the rotation are taken in
+ * fp32, the result is rounded to the storage type (round to nearest even); a token that does not move is
+ * copied bit for bit.  Values and the dimensions at and beyond rotary_dim are bit copies; rotary_dim = 0
  * is the plain compaction.  Same arguments as sharpv_kv_compact plus seq_offsets [dev] int32[num_seqs+1]
  * (the packed sequence table of sharpv_kv_calibrate_prune), rotary_dim (even, <= head_dim,
  * (rotary_dim / 2) * sizeof(element) a multiple of 16 bytes), rope_base > 0 and a workspace of

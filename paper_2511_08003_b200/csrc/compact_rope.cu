@@ -34,10 +34,17 @@ struct RopeGeom {
     int64_t row_limit;                                  // rows a source plane can hold (debug range checks)
 };
 
+// cos / sin of the rotation angle of every (kept row, rotary pair).  The angle (row's move * base^(-2i/rotary_dim))
+// is formed and reduced to [-pi, pi] in fp64 (two-constant split of 2 pi: the reduction is exact to 1e-11 for
+// moves of 10^5 positions), its sine and cosine are then taken in fp32, the precision the table is stored in.
+// The inverse frequencies are computed once per CTA.
 __global__ void __launch_bounds__(256)
 rope_table_kernel(const int32_t* __restrict__ kept_pos, const int32_t* __restrict__ kept_seq_offsets,
                   const int32_t* __restrict__ seq_offsets, int num_seqs, int64_t capacity, int half,
                   int rotary_dim, double base, float2* __restrict__ table) {
+    extern __shared__ double inv_freq[];                // [half]
+    for (int i = threadIdx.x; i < half; i += 256) inv_freq[i] = pow(base, -2.0 * (double)i / (double)rotary_dim);
+    __syncthreads();
     cudaGridDependencySynchronize();
     const int lane = threadIdx.x & 31;
     const int64_t j = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -46,11 +53,16 @@ rope_table_kernel(const int32_t* __restrict__ kept_pos, const int32_t* __restric
     const int b = upper_segment(kept_seq_offsets, num_seqs, (int)j);
     const double delta = (double)(j - __ldg(kept_seq_offsets + b)) -
                          (double)(__ldg(kept_pos + j) - __ldg(seq_offsets + b));
+    constexpr double kInvTwoPi = 0.15915494309189533577;
+    constexpr double kTwoPiHi = 6.283185307179586232;       // fl64(2 pi)
+    constexpr double kTwoPiLo = 2.4492935982947064e-16;     // 2 pi - fl64(2 pi)
     for (int i = lane; i < half; i += 32) {
-        const double ang = delta * pow(base, -2.0 * (double)i / (double)rotary_dim);
-        double sn, cs;
-        sincos(ang, &sn, &cs);
-        table[j * half + i] = make_float2((float)cs, (float)sn);
+        const double ang = delta * inv_freq[i];
+        const double turns = rint(ang * kInvTwoPi);
+        const double r = fma(-turns, kTwoPiLo, fma(-turns, kTwoPiHi, ang));
+        float sn, cs;
+        sincosf((float)r, &sn, &cs);
+        table[j * half + i] = make_float2(cs, sn);
     }
 }
 
@@ -340,7 +352,8 @@ extern "C" sharpv_status sharpv_kv_compact_rope(
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     float2* table = (float2*)workspace;
     if (rotary_dim > 0) {
-        if (launch_dependent(rope_table_kernel, dim3((unsigned)((capacity + 7) / 8)), dim3(256), 0, stream, kept_pos,
+        if (launch_dependent(rope_table_kernel, dim3((unsigned)((capacity + 7) / 8)), dim3(256),
+                             (size_t)g.half * sizeof(double), stream, kept_pos,
                              kept_seq_offsets, seq_offsets, (int)num_seqs, capacity, g.half, (int)rotary_dim,
                              rope_base, table) != cudaSuccess) {
             (void)cudaGetLastError();

@@ -380,7 +380,11 @@ template <int DT>
 __global__ void __launch_bounds__(kFinThreads)
 score_finalize_kernel(const FusedParams p) {
     __shared__ float4 g_sum[4][kMaxTokensFused];
-    __shared__ float f_s2[kMaxTokensFused], f_t2[kMaxTokensFused], f_aa[kMaxTokensFused], f_bb[kMaxTokensFused];
+    __shared__ float f_all[4 * kMaxTokensFused];        // four per-row arrays, later the four partial ranks
+    float* const f_s2 = f_all;
+    float* const f_t2 = f_all + kMaxTokensFused;
+    float* const f_aa = f_all + 2 * kMaxTokensFused;
+    float* const f_bb = f_all + 3 * kMaxTokensFused;
     __shared__ int f_fl[kMaxTokensFused];
     __shared__ float red[kFinThreads / 32 + 1];     // also the scratch of the block scan
     const int t = blockIdx.x;
@@ -486,14 +490,24 @@ score_finalize_kernel(const FusedParams p) {
         comp[tid] = tid < p.f ? mine : 0ull;
     }
     __syncthreads();
+    // all four groups of 256 threads count: group q compares token `row` with the keys q, q+4, ... of the
+    // frame (as pairs), the four partial ranks meet in shared memory
+    int* ranks = reinterpret_cast<int*>(f_all);         // [4][256]; the per-row arrays were last read barriers ago
+    const unsigned long long my_key = row < p.f ? comp[row] : ~0ull;
+    {
+        int part = 0;
+        const int fpad = (p.f + 1) & ~1;
+        for (int j2 = 2 * grp; j2 < fpad; j2 += 8) {
+            const ulonglong2 c2 = *reinterpret_cast<const ulonglong2*>(comp + j2);
+            part += (c2.x > my_key) + (c2.y > my_key);
+        }
+        ranks[grp * kMaxTokensFused + row] = part;
+    }
+    __syncthreads();
     int keep = 0;
     if (tid < p.f && kt > 0) {
-        int rank = 0;
-        const int fpad = (p.f + 1) & ~1;
-        for (int j2 = 0; j2 < fpad; j2 += 2) {
-            const ulonglong2 c2 = *reinterpret_cast<const ulonglong2*>(comp + j2);
-            rank += (c2.x > mine) + (c2.y > mine);
-        }
+        const int rank = (ranks[tid] + ranks[kMaxTokensFused + tid]) +
+                         (ranks[2 * kMaxTokensFused + tid] + ranks[3 * kMaxTokensFused + tid]);
         keep = rank < kt;
     }
     int total;
