@@ -18,6 +18,8 @@
 
 #include <cuda_bf16.h>
 
+#include <cmath>
+
 namespace sharpv {
 namespace {
 
@@ -41,9 +43,9 @@ struct RopeGeom {
 __global__ void __launch_bounds__(256)
 rope_table_kernel(const int32_t* __restrict__ kept_pos, const int32_t* __restrict__ kept_seq_offsets,
                   const int32_t* __restrict__ seq_offsets, int num_seqs, int64_t capacity, int half,
-                  int rotary_dim, double base, float2* __restrict__ table) {
-    extern __shared__ double inv_freq[];                // [half]
-    for (int i = threadIdx.x; i < half; i += 256) inv_freq[i] = pow(base, -2.0 * (double)i / (double)rotary_dim);
+                  int rotary_dim, double log_base, float2* __restrict__ table) {
+    extern __shared__ double inv_freq[];                // [half]: base^(-2i/rotary_dim) = exp(-(2i/rotary_dim) ln base)
+    for (int i = threadIdx.x; i < half; i += 256) inv_freq[i] = exp(-2.0 * (double)i / (double)rotary_dim * log_base);
     __syncthreads();
     cudaGridDependencySynchronize();
     const int lane = threadIdx.x & 31;
@@ -355,7 +357,7 @@ extern "C" sharpv_status sharpv_kv_compact_rope(
         if (launch_dependent(rope_table_kernel, dim3((unsigned)((capacity + 7) / 8)), dim3(256),
                              (size_t)g.half * sizeof(double), stream, kept_pos,
                              kept_seq_offsets, seq_offsets, (int)num_seqs, capacity, g.half, (int)rotary_dim,
-                             rope_base, table) != cudaSuccess) {
+                             log(rope_base), table) != cudaSuccess) {
             (void)cudaGetLastError();
             return SHARPV_ERR_CUDA;
         }
