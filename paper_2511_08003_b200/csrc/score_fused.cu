@@ -34,7 +34,6 @@ constexpr int kMaxVisits = 8;           // rows a lane group walks per tile
 constexpr int kMaxTokensFused = 256;    // the finaliser takes one row per thread of a 256-thread group
 static_assert(4 * kMaxWarps * kMaxVisits >= kMaxTokensFused, "the warps must cover the largest frame");
 constexpr int kRedStride = 9;           // floats per (visit, row) slot of a warp's patch: 8 lane parts + 1 pad
-constexpr int kFinThreads = 1024;
 
 struct FusedParams {
     const char* tokens;
@@ -374,12 +373,15 @@ score_pass_kernel(const FusedParams p) {
 }
 
 // One CTA per frame: adds the slices in a fixed order, writes S, T, I, ratio_t and k_t.
-// 1024 threads = 4 groups x 256 rows; group q adds slices q, q+4, ... (up to 8 records in flight per
-// thread), then the four group sums are added in order.
-template <int DT>
-__global__ void __launch_bounds__(kFinThreads)
+// G groups of 256 rows; group q adds slices q, q+G, ... (up to 8 records in flight per thread), then the
+// group sums are added in order.  G = 4 (1024 threads, one CTA on an SM) is the quickest for a frame;
+// G = 2 (512 threads, two CTAs on an SM) takes twice the frames at a time and is used when there are
+// more frames than SMs.
+template <int DT, int G>
+__global__ void __launch_bounds__(256 * G, G == 2 ? 2 : 0)
 score_finalize_kernel(const FusedParams p) {
-    __shared__ float4 g_sum[4][kMaxTokensFused];
+    constexpr int kFinThreads = 256 * G;
+    __shared__ float4 g_sum[G][kMaxTokensFused];
     __shared__ float f_all[4 * kMaxTokensFused];        // four per-row arrays, later the four partial ranks
     float* const f_s2 = f_all;
     float* const f_t2 = f_all + kMaxTokensFused;
@@ -398,11 +400,11 @@ score_finalize_kernel(const FusedParams p) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);       // ||a||^2, <a, mean>, ||a - b||^2, ||b||^2
     float sm = 0.f;
     const float4* src = p.part + ((int64_t)t * p.nsl) * p.f + row;
-    for (int s0 = grp; s0 < p.nsl; s0 += 32) {
+    for (int s0 = grp; s0 < p.nsl; s0 += 8 * G) {
         float4 q[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const int s = s0 + 4 * i;
+            const int s = s0 + G * i;
             q[i] = (row < p.f && s < p.nsl) ? __ldcg(src + (int64_t)s * p.f) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         if (s0 == grp) {
@@ -423,9 +425,15 @@ score_finalize_kernel(const FusedParams p) {
     for (int i = 0; i < kFinThreads / 32; ++i) smm += red[i];
 
     if (tid < p.f) {
-        const float4 a0 = g_sum[0][tid], a1 = g_sum[1][tid], a2 = g_sum[2][tid], a3 = g_sum[3][tid];
-        const float aa = (a0.x + a1.x) + (a2.x + a3.x), am = (a0.y + a1.y) + (a2.y + a3.y);
-        const float db = (a0.z + a1.z) + (a2.z + a3.z), bb = (a0.w + a1.w) + (a2.w + a3.w);
+        float aa, am, db, bb;
+        if constexpr (G == 4) {
+            const float4 a0 = g_sum[0][tid], a1 = g_sum[1][tid], a2 = g_sum[2][tid], a3 = g_sum[3][tid];
+            aa = (a0.x + a1.x) + (a2.x + a3.x); am = (a0.y + a1.y) + (a2.y + a3.y);
+            db = (a0.z + a1.z) + (a2.z + a3.z); bb = (a0.w + a1.w) + (a2.w + a3.w);
+        } else {
+            const float4 a0 = g_sum[0][tid], a1 = g_sum[1][tid];
+            aa = a0.x + a1.x; am = a0.y + a1.y; db = a0.z + a1.z; bb = a0.w + a1.w;
+        }
         const float s2 = dissim_sq_from_dot(aa, smm, am);
         const float t2 = is_first ? 0.f : dissim_sq_from_sums(aa, bb, db);      // a video's first frame: db, bb unused
         int fl = 0;
@@ -490,14 +498,14 @@ score_finalize_kernel(const FusedParams p) {
         comp[tid] = tid < p.f ? mine : 0ull;
     }
     __syncthreads();
-    // all four groups of 256 threads count: group q compares token `row` with the keys q, q+4, ... of the
-    // frame (as pairs), the four partial ranks meet in shared memory
-    int* ranks = reinterpret_cast<int*>(f_all);         // [4][256]; the per-row arrays were last read barriers ago
+    // all groups of 256 threads count: group q compares token `row` with the keys q, q+G, ... of the
+    // frame (as pairs), the partial ranks meet in shared memory
+    int* ranks = reinterpret_cast<int*>(f_all);         // [G][256]; the per-row arrays were last read barriers ago
     const unsigned long long my_key = row < p.f ? comp[row] : ~0ull;
     {
         int part = 0;
         const int fpad = (p.f + 1) & ~1;
-        for (int j2 = 2 * grp; j2 < fpad; j2 += 8) {
+        for (int j2 = 2 * grp; j2 < fpad; j2 += 2 * G) {
             const ulonglong2 c2 = *reinterpret_cast<const ulonglong2*>(comp + j2);
             part += (c2.x > my_key) + (c2.y > my_key);
         }
@@ -506,8 +514,8 @@ score_finalize_kernel(const FusedParams p) {
     __syncthreads();
     int keep = 0;
     if (tid < p.f && kt > 0) {
-        const int rank = (ranks[tid] + ranks[kMaxTokensFused + tid]) +
-                         (ranks[2 * kMaxTokensFused + tid] + ranks[3 * kMaxTokensFused + tid]);
+        int rank = ranks[tid] + ranks[kMaxTokensFused + tid];
+        if constexpr (G == 4) rank += ranks[2 * kMaxTokensFused + tid] + ranks[3 * kMaxTokensFused + tid];
         keep = rank < kt;
     }
     int total;
@@ -627,8 +635,10 @@ sharpv_status launch(const FusedScoreArgs& a, FusedParams& p, int dev, int sms) 
         return SHARPV_ERR_CUDA;
     }
     // the finaliser starts while the pass drains and waits for it with cudaGridDependencySynchronize
-    if (launch_dependent(score_finalize_kernel<DT>, dim3((unsigned)a.F), dim3(kFinThreads), 0, a.stream, p) !=
-        cudaSuccess) {
+    const cudaError_t fin = a.F > sms
+        ? launch_dependent(score_finalize_kernel<DT, 2>, dim3((unsigned)a.F), dim3(512), 0, a.stream, p)
+        : launch_dependent(score_finalize_kernel<DT, 4>, dim3((unsigned)a.F), dim3(1024), 0, a.stream, p);
+    if (fin != cudaSuccess) {
         (void)cudaGetLastError();
         return SHARPV_ERR_CUDA;
     }
