@@ -876,6 +876,44 @@ def test_prune_frames_random_shapes_ties_and_capacity(seed):
         assert "tokens" not in small
 
 
+@pytest.mark.parametrize("F,f,bf16", [(149, 40, True), (300, 196, True), (700, 9, False), (5000, 6, True)])
+def test_prune_frames_with_more_frames_than_sms(F, f, bf16):
+    """Stage one in one call on batches with more frames than the GPU has SMs (the finaliser then runs as
+    two smaller CTAs per SM) and with more frames than a CTA scans by itself (the kept lists' offsets then
+    come from the one-CTA scan kernel): scores against the oracle, selection and gather exact on the GPU's
+    own scores, several videos, ties, and a capacity below the kept count."""
+    rng = np.random.default_rng(9000 + F)
+    d = 128 if bf16 else 64
+    cuts = np.sort(rng.choice(np.arange(1, F), size=5, replace=False))
+    vfo = np.concatenate([[0], cuts, [F]]).astype(np.int32)
+    x = rng.standard_normal((F * f, d)).astype(np.float32)
+    for t in range(1, F):
+        x[t * f:(t + 1) * f] = 0.9 * x[(t - 1) * f:t * f] + 0.436 * x[t * f:(t + 1) * f]
+    x[3 * f:4 * f] = x[3 * f]                                      # a frame of identical tokens: every score ties
+    xs = W.f32_to_bf16_bits(x) if bf16 else x
+    o = orc.score_frames(xs, vfo, f, w=1.0, min_keep=1, nthreads=NT)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    g = sv.sharpv_prune_frames(to_dev(xs), torch.from_numpy(vfo).cuda(), F, f, w=1.0, min_keep=1, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert_scores(g, o, f, keys=("importance", "ratio"))
+    k_gpu = to_host(g["k"])
+    check_budgets(k_gpu, o, f)
+    idx_o, off_o = orc.select_tokens(to_host(g["importance"]), k_gpu, f)
+    n = int(g["num_kept"].item())
+    assert n == idx_o.size
+    np.testing.assert_array_equal(to_host(g["kept_offsets"]), off_o)
+    np.testing.assert_array_equal(to_host(g["kept_index"])[:n], idx_o)
+    np.testing.assert_array_equal(to_host(g["tokens"])[:n], orc.gather_rows(xs, idx_o))
+    cap = n // 3
+    small = sv.sharpv_prune_frames(to_dev(xs), torch.from_numpy(vfo).cuda(), F, f, w=1.0, min_keep=1, capacity=cap,
+                                   status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == sv.Status.ERR_CAPACITY and int(small["num_kept"].item()) == n
+    np.testing.assert_array_equal(to_host(small["kept_index"])[:cap], idx_o[:cap])
+    np.testing.assert_array_equal(to_host(small["tokens"])[:cap], orc.gather_rows(xs, idx_o[:cap]))
+
+
 def test_many_frames_and_many_positions_use_the_scan_kernels():
     """Batches beyond the sizes at which every CTA adds up the counts in front of it itself: 20,000 tiny
     frames through the selection, 1.2 million packed positions through the calibration (their offsets then
