@@ -37,6 +37,11 @@ struct LayerStrides {
 
 constexpr int kRowsPerCta = 4;          // one packed position per warp; small CTAs balance the SMs
 constexpr int64_t kInlineBaseChunks = 4096;  // up to this many chunks every chunk CTA adds up the counts in front of it itself
+// Up to this many positions no chunk counts are kept at all: a chunk CTA counts the keep flags in front
+// of it (one byte a position, 16 to a load, L2-resident), which saves clearing the counters and the
+// atomics that fill them.  The cost grows with the square of the positions, hence the limit.
+constexpr int64_t kCountFlagsPositions = 65536;
+enum BaseSource { kBaseFromCounts = 0, kBaseFromScan = 1, kBaseFromFlags = 2 };
 
 template <int DT>
 __global__ void __launch_bounds__(kRowsPerCta * 32)
@@ -108,7 +113,7 @@ calibrate_cos_kernel(const char* __restrict__ hidden, int64_t hidden_row_bytes,
     }
     if (lane == 0 && flags) {
         flags[p] = (uint8_t)keep;
-        if (keep) atomicAdd(chunk_counts + p / kChunk, 1);     // integer: order does not matter
+        if (keep && chunk_counts) atomicAdd(chunk_counts + p / kChunk, 1);     // integer: order does not matter
     }
 }
 
@@ -121,7 +126,7 @@ write_kept_kernel(const uint8_t* __restrict__ flags, const int32_t* __restrict__
     __shared__ int s_base;
     const int c = blockIdx.x;
     flags += (int64_t)blockIdx.y * ls.flags;
-    chunk_counts += (int64_t)blockIdx.y * ls.chunks;
+    if (chunk_counts) chunk_counts += (int64_t)blockIdx.y * ls.chunks;
     out_kept_pos += (int64_t)blockIdx.y * ls.kept;
     out_kept_seq_offsets += (int64_t)blockIdx.y * ls.offsets;
     cudaGridDependencySynchronize();        // flags and chunk counts come from the kernel in front
@@ -129,10 +134,22 @@ write_kept_kernel(const uint8_t* __restrict__ flags, const int32_t* __restrict__
     const int64_t p = (int64_t)c * kChunk + threadIdx.x;
     const int keep = p < T ? flags[p] : 0;
     // kept positions before this chunk: the counts of the chunks in front, or (many chunks) their
-    // exclusive scan, which a one-CTA kernel in front has left in the same array
+    // exclusive scan, which a one-CTA kernel in front has left in the same array, or (few positions, no
+    // counts kept) the keep flags in front, counted here
     int part = 0;
-    if (bases_ready) {
+    if (bases_ready == kBaseFromScan) {
         if (threadIdx.x == 0) part = chunk_counts[c];
+    } else if (bases_ready == kBaseFromFlags) {
+        const uint4* fv = reinterpret_cast<const uint4*>(flags);       // flags are 0 or 1: byte sums by dp4a
+        unsigned acc = 0;
+        for (int i = threadIdx.x; i < c * (kChunk / 16); i += kChunk) {
+            const uint4 w = __ldcg(fv + i);
+            acc = __dp4a(w.x, 0x01010101u, acc);
+            acc = __dp4a(w.y, 0x01010101u, acc);
+            acc = __dp4a(w.z, 0x01010101u, acc);
+            acc = __dp4a(w.w, 0x01010101u, acc);
+        }
+        part = (int)acc;
     } else {
         for (int i = threadIdx.x; i < c; i += kChunk) part += chunk_counts[i];
     }
@@ -237,8 +254,12 @@ static sharpv_status calibrate_impl(
     const unsigned chunks = (unsigned)num_chunks(total_seq_tokens);
     const unsigned ctas = (unsigned)((total_seq_tokens + kRowsPerCta - 1) / kRowsPerCta);
     const int nvec = d * eb / 16;
+    const int bases_ready = total_seq_tokens <= kCountFlagsPositions ? kBaseFromFlags
+                            : (int64_t)chunks > kInlineBaseChunks     ? kBaseFromScan
+                                                                      : kBaseFromCounts;
+    if (bases_ready == kBaseFromFlags) chunk_counts = nullptr;
     // the per-chunk counts are accumulated with atomics and must start at zero
-    if (cudaMemsetAsync(chunk_counts, 0, sizeof(int32_t) * (size_t)chunks, stream) != cudaSuccess)
+    if (chunk_counts && cudaMemsetAsync(chunk_counts, 0, sizeof(int32_t) * (size_t)chunks, stream) != cudaSuccess)
         return SHARPV_ERR_CUDA;
     {
         auto kern = dtype == SHARPV_F32 ? calibrate_cos_kernel<SHARPV_F32> : calibrate_cos_kernel<SHARPV_BF16>;
@@ -250,8 +271,7 @@ static sharpv_status calibrate_impl(
             return SHARPV_ERR_CUDA;
         }
     }
-    const int bases_ready = (int64_t)chunks > kInlineBaseChunks;
-    if (bases_ready &&
+    if (bases_ready == kBaseFromScan &&
         launch_dependent(exclusive_scan_i32_kernel<false>, dim3(1), dim3(kScanThreads), 0, stream,
                          (const int32_t*)chunk_counts, (int64_t)chunks, 0, chunk_counts, (int32_t*)nullptr,
                          (int32_t*)nullptr, (int64_t)-1, (int32_t*)nullptr) != cudaSuccess) {
@@ -439,7 +459,9 @@ extern "C" sharpv_status sharpv_kv_prune_layers(
     const unsigned ctas = (unsigned)((total_seq_tokens + kRowsPerCta - 1) / kRowsPerCta);
     const int nvec = (int)(d * eb / 16);
     if (n_layers > 65535) return SHARPV_ERR_UNSUPPORTED;
-    if (per_token) {
+    const bool count_flags = total_seq_tokens <= kCountFlagsPositions;
+    if (count_flags) chunk_counts = nullptr;
+    if (per_token && !count_flags) {
         // every layer's chunk counters start at zero (they sit `one` bytes apart: clear the whole range)
         if (cudaMemsetAsync(workspace, 0, one * (size_t)n_layers, stream) != cudaSuccess) return SHARPV_ERR_CUDA;
     }
@@ -456,7 +478,8 @@ extern "C" sharpv_status sharpv_kv_prune_layers(
     }
     if (per_token) {
         if (launch_dependent(write_kept_kernel, dim3(chunks, (unsigned)n_layers), dim3(kChunk), 0, stream,
-                             (const uint8_t*)flags, (const int32_t*)chunk_counts, 0, total_seq_tokens, num_seqs,
+                             (const uint8_t*)flags, (const int32_t*)chunk_counts,
+                             (int)(count_flags ? kBaseFromFlags : kBaseFromCounts), total_seq_tokens, num_seqs,
                              seq_offsets, capacity, out_kept_pos, out_kept_seq_offsets, status_word, ls) !=
             cudaSuccess) {
             (void)cudaGetLastError();
