@@ -1084,7 +1084,8 @@ def _device_kv(wl, seed):
 def test_full_size_workloads(name):
     """The 16-video ragged batch (424 frames) and the 256-frame video at their full sizes: scores,
     budgets and kept sets element by element against the oracle; compacted K/V (4.8 GB / 2.9 GB) on
-    sampled planes and rows plus properties that hold for every plane."""
+    sampled planes and rows plus properties that hold for every plane; then the single-call stage one, the
+    rotary and the in-place compaction on the same inputs."""
     wl = W.PRESETS[name]()
     W.fill_tokens(wl)
     W.fill_hidden(wl)
@@ -1138,3 +1139,40 @@ def test_full_size_workloads(name):
     kept_d = gc["kept_pos"][:nk].long()
     assert torch.equal(dst[:, :, :, :nk].view(torch.int16), kv[:, :, :, kept_d].view(torch.int16))
     assert int(dst[:, :, :, nk:].view(torch.int16).abs().max().item()) == 0
+
+    # stage one in one call at the full size: bit for bit the two calls above
+    pr = sv.sharpv_prune_frames(dw.tokens, dw.video_frame_offsets, F, f)
+    torch.cuda.synchronize()
+    assert torch.equal(pr["importance"], g["importance"]) and torch.equal(pr["k"], g["k"])
+    assert int(pr["num_kept"].item()) == n and torch.equal(pr["kept_offsets"], sel["kept_offsets"])
+    assert torch.equal(pr["kept_index"][:n], sel["kept_index"][:n])
+    assert torch.equal(pr["tokens"][:n].view(torch.int16), sel["tokens"][:n].view(torch.int16))
+    del pr, sel
+
+    # rotary re-encoding at the full size: values and the keys that do not move are bit copies of the plain
+    # compaction; sampled key planes against the oracle
+    seqs = torch.from_numpy(wl.seq_offsets).cuda()
+    dst.zero_()
+    sv.sharpv_kv_compact_rope(kv, dst, gc["kept_pos"], gc["kept_seq_offsets"], seqs, T, Dh, 1.0e6)
+    torch.cuda.synchronize()
+    assert torch.equal(dst[:, 1, :, :nk].view(torch.int16), kv[:, 1][:, :, kept_d].view(torch.int16))
+    assert int(dst[:, :, :, nk:].view(torch.int16).abs().max().item()) == 0
+    b_of = np.searchsorted(wl.seq_offsets, kept, side="right") - 1
+    still = np.nonzero(kept - wl.seq_offsets[b_of] == np.arange(nk) - kso[b_of])[0]
+    still_d = torch.from_numpy(still).cuda()
+    assert torch.equal(dst[:, 0][:, :, still_d].view(torch.int16), kv[:, 0][:, :, kept_d[still_d]].view(torch.int16))
+    for (l, _, h) in sorted(planes)[:3]:
+        src5 = np.ascontiguousarray(to_host(kv[l, :, h])[None, :, None])          # [1, 2, 1, T, Dh]
+        want = orc.kv_compact_rope(src5, kept, kso, wl.seq_offsets, Dh, 1.0e6)[0, 0, 0]
+        got = W.bf16_bits_to_f32(to_host(dst[l, 0, h, :nk])).astype(np.float64)
+        pair = np.hypot(want[:, :Dh // 2], want[:, Dh // 2:])
+        pair = np.concatenate([pair, pair], axis=-1)
+        assert np.all(np.abs(got - want) <= 2.0 ** -8 * np.abs(want) * 1.001 + 4e-6 * pair + 1e-30)
+
+    # in place at the full size: the kept prefix of every plane equals the rows gathered from the original,
+    # the tail keeps its old contents
+    dst.copy_(kv)
+    sv.sharpv_kv_compact(dst, dst, gc["kept_pos"], gc["kept_seq_offsets"], capacity=T)
+    torch.cuda.synchronize()
+    assert torch.equal(dst[:, :, :, :nk].view(torch.int16), kv[:, :, :, kept_d].view(torch.int16))
+    assert torch.equal(dst[:, :, :, nk:].view(torch.int16), kv[:, :, :, nk:].view(torch.int16))
