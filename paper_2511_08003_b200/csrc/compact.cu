@@ -2,8 +2,8 @@
 // of the kept positions are copied, in order, to a dense prefix of the destination plane.
 // One index list serves all planes.
 //
-// Out of place: persistent CTAs walk the (plane, tile) list with 128-bit loads and stores through
-// registers.  In place (kv_dst == kv_src): one CTA per plane, front to back.
+// Out of place: one short-lived CTA per (row tile, plane) with 128-bit loads and stores through
+// registers.  In place (kv_dst == kv_src): the rows are split into levels of disjoint row ranges (below).
 // Bulk async copies (one cp.async.bulk per kept 256-byte row into a shared-memory tile, one bulk
 // store per dense tile) were measured and lost: the copy engine's per-request cost caps 256-byte
 // rows near 2.2 TB/s of reads, against 2.7 TB/s for this kernel at the same kept share.
@@ -15,94 +15,64 @@ namespace {
 
 constexpr int kCompactThreads = 256;
 constexpr int kCompactUnroll = 4;         // 16-byte vectors in flight per thread
-constexpr int kCompactCtasPerSm = 5;      // resident CTAs per SM at 47 registers
+constexpr int kCompactCtasPerSm = 5;      // resident CTAs per SM of the in-place level kernel (47 registers)
+constexpr int kGatherCtasPerSm = 8;       // of the out-of-place kernel: 32 registers, every thread slot of an SM taken
+constexpr int kGatherTilesPerCta = 2;     // row tiles a CTA takes at least when the list is as long as `capacity`
+constexpr int64_t kGatherMaxCtas = 32768; // CTAs of one launch (many times the 148 x 8 that are resident)
 
 struct PlaneGeom {
     int64_t src_layer, src_kv, src_head, src_token;     // bytes
     int64_t dst_layer, dst_kv, dst_head, dst_token;     // bytes
     int num_kv_heads, layer_begin, row_vecs;            // row_vecs = 16-byte vectors per row
+    int row_shift;                                      // log2(row_vecs) if that is a power of two, else -1
     int64_t row_limit;                                  // rows a source plane can hold (what a dense layout implies)
 };
 
-// Persistent CTAs share the (plane, tile) list in contiguous runs; a tile is tile_rows destination rows.
-// Each thread moves kUnroll 16-byte vectors per tile, all loads issued before the first store.
+// One CTA per (row tile, plane): tile_rows destination rows of one plane; blockIdx.y is the plane.  Each
+// thread moves kUnroll 16-byte vectors, all loads issued before the first store.  The grid is laid out for
+// `capacity` rows (the kept count is only known on the device) with kGatherTilesPerCta tiles to a CTA; a CTA
+// whose tile starts behind the kept count leaves at once.  CTAs that come and go keep reads and writes of
+// the SMs mixed: persistent CTAs walking the same tiles in step stay about 10 % under it.
 template <int kUnroll, bool kPerLayer>
-__global__ void __launch_bounds__(kCompactThreads, kCompactCtasPerSm)
-kv_compact_kernel(const char* __restrict__ src, char* __restrict__ dst, PlaneGeom g, int planes,
+__global__ void __launch_bounds__(kCompactThreads, kGatherCtasPerSm)
+kv_compact_kernel(const char* __restrict__ src, char* __restrict__ dst, PlaneGeom g,
                   const int32_t* __restrict__ kept_pos, const int32_t* __restrict__ n_kept_ptr,
                   int64_t kept_stride, int64_t count_stride, int64_t capacity, int32_t* status_word) {
-    cudaGridDependencySynchronize();        // the index list and the cache come from earlier work on the stream
-    // One list for all layers (strides 0), or every layer of the range its own list and count; then the
-    // tile grid is laid out for `capacity` rows and a tile beyond its layer's count is skipped.
-    constexpr bool per_layer = kPerLayer;
-    int64_t n = capacity;
-    if (!per_layer) {
-        const int64_t n_all = __ldg(n_kept_ptr);
-        if (blockIdx.x == 0 && threadIdx.x == 0 && n_all > capacity) report(status_word, SHARPV_ERR_CAPACITY);
-        n = min(n_all, capacity);
-    }
-    if (n <= 0) return;
+    const int plane = blockIdx.y;
+    const int li = plane / (2 * g.num_kv_heads), kv = (plane / g.num_kv_heads) & 1, h = plane % g.num_kv_heads;
     const int tile_rows = kCompactThreads * kUnroll / g.row_vecs;      // >= 1, checked by the host
-    const int64_t tiles_per_plane = (n + tile_rows - 1) / tile_rows;
-    const int64_t total_tiles = tiles_per_plane * planes;
-    // Every CTA takes a contiguous run of tiles in (plane, row tile) order: it writes one dense stretch of
-    // a plane after the other, and where it stands (plane, layer, K|V, head, row tile) is stepped, not
-    // divided out again for every tile.
-    const int64_t t0 = blockIdx.x, t1 = total_tiles;
-    if (t0 >= t1) return;
-    // tiles are dealt out round robin; the step from one tile of this CTA to its next is a fixed number
-    // of planes and row tiles, so where the CTA stands is stepped, not divided out again
-    const int step_planes = (int)(gridDim.x / tiles_per_plane);
-    const int64_t step_rt = gridDim.x - (int64_t)step_planes * tiles_per_plane;
-    int plane = (int)(t0 / tiles_per_plane);
-    int64_t rt = t0 - (int64_t)plane * tiles_per_plane;
-    // what a thread moves in every tile: vector vv of row rr of the tile
-    int rr[kUnroll];
-    int64_t voff[kUnroll];
+    cudaGridDependencySynchronize();        // the index list and the cache come from earlier work on the stream
+    // One list for all layers (strides 0), or every layer of the range its own list and count.
+    const int32_t* list = kPerLayer ? kept_pos + li * kept_stride : kept_pos;
+    const int64_t n_all = __ldg(n_kept_ptr + (kPerLayer ? li * count_stride : 0));
+    if (blockIdx.x == 0 && threadIdx.x == 0 && kv == 0 && h == 0 && (kPerLayer || li == 0) && n_all > capacity)
+        report(status_word, SHARPV_ERR_CAPACITY);
+    const int64_t n = min(n_all, capacity);
+    const char* s = src + (g.layer_begin + li) * g.src_layer + kv * g.src_kv + h * g.src_head;
+    char* o = dst + (g.layer_begin + li) * g.dst_layer + kv * g.dst_kv + h * g.dst_head;
+    // the grid holds a fraction of the row tiles `capacity` rows would need: a CTA takes tile blockIdx.x,
+    // then blockIdx.x + gridDim.x, ... while they start in front of the kept count
+    for (int64_t row0 = (int64_t)blockIdx.x * tile_rows; row0 < n; row0 += (int64_t)gridDim.x * tile_rows) {
+        uint4 r[kUnroll];
+        unsigned moved = 0;                 // bit u: vector u of this thread is copied
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-        const int q = threadIdx.x + u * kCompactThreads;
-        rr[u] = q / g.row_vecs;
-        voff[u] = (int64_t)(q - rr[u] * g.row_vecs) * 16;
-    }
-    for (int64_t tile = t0; tile < t1; tile += gridDim.x) {
-        const int64_t row0 = rt * tile_rows;
-        const int li = plane / (2 * g.num_kv_heads), kv = (plane / g.num_kv_heads) & 1, h = plane % g.num_kv_heads;
-        const int32_t* list = per_layer ? kept_pos + li * kept_stride : kept_pos;
-        bool skip = false;
-        if (per_layer) {
-            const int64_t n_all = __ldg(n_kept_ptr + li * count_stride);
-            if (row0 == 0 && kv == 0 && h == 0 && threadIdx.x == 0 && n_all > capacity)
-                report(status_word, SHARPV_ERR_CAPACITY);
-            n = min(n_all, capacity);
-            skip = row0 >= n;
-        }
-        if (!skip) {
-            const char* s = src + (g.layer_begin + li) * g.src_layer + kv * g.src_kv + h * g.src_head;
-            char* o = dst + (g.layer_begin + li) * g.dst_layer + kv * g.dst_kv + h * g.dst_head;
-            uint4 r[kUnroll];
-            int64_t off[kUnroll];
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                const int64_t j = row0 + rr[u];
-                off[u] = -1;
-                if (rr[u] < tile_rows && j < n) {
-                    const int64_t from = __ldg(list + j);
-                    if (index_ok(from >= 0 && from < g.row_limit, status_word)) {
-                        r[u] = ld_stream(s + from * g.src_token + voff[u]);
-                        off[u] = j * g.dst_token + voff[u];
-                    }
+        for (int u = 0; u < kUnroll; ++u) {
+            const int q = threadIdx.x + u * kCompactThreads;
+            const int rr = g.row_shift >= 0 ? q >> g.row_shift : q / g.row_vecs;      // row of the tile, vector of the row
+            const int64_t j = row0 + rr;
+            if (rr < tile_rows && j < n) {
+                const int64_t from = __ldg(list + j);
+                if (index_ok(from >= 0 && from < g.row_limit, status_word)) {
+                    r[u] = ld_stream(s + from * g.src_token + (int64_t)(q - rr * g.row_vecs) * 16);
+                    moved |= 1u << u;
                 }
             }
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u)
-                if (off[u] >= 0) st_stream(o + off[u], r[u]);
         }
-        plane += step_planes;
-        rt += step_rt;
-        if (rt >= tiles_per_plane) {
-            rt -= tiles_per_plane;
-            ++plane;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int q = threadIdx.x + u * kCompactThreads;
+            const int rr = g.row_shift >= 0 ? q >> g.row_shift : q / g.row_vecs;
+            if (moved >> u & 1) st_stream(o + (row0 + rr) * g.dst_token + (int64_t)(q - rr * g.row_vecs) * 16, r[u]);
         }
     }
 }
@@ -336,6 +306,9 @@ sharpv_status kv_compact_launch(const void* kv_src, const sharpv_kv_layout* src_
     g.layer_begin = layer_begin;
     g.row_vecs = (int)(src_layout->head_dim * eb / 16);
     g.row_limit = kv_row_limit(src_layout);
+    g.row_shift = -1;
+    for (int b = 0; b < 31; ++b)
+        if (g.row_vecs == 1 << b) g.row_shift = b;
     if (g.row_vecs > kCompactThreads * kCompactUnroll) return SHARPV_ERR_UNSUPPORTED;    // rows over 16 KB
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -365,8 +338,13 @@ sharpv_status kv_compact_launch(const void* kv_src, const sharpv_kv_layout* src_
         return SHARPV_OK;
     }
     auto kern = count_stride != 0 ? kv_compact_kernel<kCompactUnroll, true> : kv_compact_kernel<kCompactUnroll, false>;
-    if (launch_dependent(kern, dim3(grid), dim3(kCompactThreads), 0, stream,
-                         (const char*)kv_src, (char*)kv_dst, g, planes, kept_pos, n_kept_ptr, kept_stride,
+    // at most kGatherMaxCtas CTAs in all: with a list much shorter than `capacity` most of them only look
+    // at the count and leave, and that has to stay cheap
+    int64_t row_tiles = ((capacity + tile_rows - 1) / tile_rows + kGatherTilesPerCta - 1) / kGatherTilesPerCta;
+    const int64_t most = kGatherMaxCtas / planes > 1 ? kGatherMaxCtas / planes : 1;
+    if (row_tiles > most) row_tiles = most;
+    if (launch_dependent(kern, dim3((unsigned)row_tiles, (unsigned)planes), dim3(kCompactThreads), 0, stream,
+                         (const char*)kv_src, (char*)kv_dst, g, kept_pos, n_kept_ptr, kept_stride,
                          count_stride, capacity, status_word) != cudaSuccess) {
         (void)cudaGetLastError();
         return SHARPV_ERR_CUDA;
