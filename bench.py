@@ -45,9 +45,9 @@ LAUNCHES_PER_STEP = {"prune": 3, "score": 2, "select": 2, "calibrate": 2, "compa
 # used only when the run reproduces the captured launch (same workload, threshold, kept count, plain
 # out-of-place compaction); `commit` is the source revision the counters were taken on.
 NCU_TRAFFIC = {
-    # 8 of the 28 layers captured (1.65 GB on the device): 354,548,224 B read + 305,405,440 B written, scaled by
-    # 28 / 8.  Reads equal the algorithmic reads; about 49 MB of writes were still in L2 when the kernel ended.
-    ("long_video", "compact"): {"bytes": 2_309_837_824, "M": 0.788, "kept_stage_two": 21633, "commit": "4d130b1"},
+    # 8 of the 28 layers captured (1.65 GB on the device): 354,534,400 B read + 304,179,456 B written, scaled by
+    # 28 / 8.  Reads equal the algorithmic reads; about 50 MB of writes were still in L2 when the kernel ended.
+    ("long_video", "compact"): {"bytes": 2_305_498_496, "M": 0.788, "kept_stage_two": 21633, "commit": "9281fd8"},
 }
 
 
