@@ -37,15 +37,19 @@ template <int kUnroll, bool kPerLayer>
 __global__ void __launch_bounds__(kCompactThreads, kGatherCtasPerSm)
 kv_compact_kernel(const char* __restrict__ src, char* __restrict__ dst, PlaneGeom g,
                   const int32_t* __restrict__ kept_pos, const int32_t* __restrict__ n_kept_ptr,
-                  int64_t kept_stride, int64_t count_stride, int64_t capacity, int32_t* status_word) {
+                  int64_t kept_stride, int64_t count_stride, int64_t capacity, int kv_only, int32_t* status_word) {
+    // blockIdx.y counts the planes of the call: (layer, K|V, head), or (layer, head) of the keys / the values alone
     const int plane = blockIdx.y;
-    const int li = plane / (2 * g.num_kv_heads), kv = (plane / g.num_kv_heads) & 1, h = plane % g.num_kv_heads;
+    const int h = plane % g.num_kv_heads;
+    const int li = kv_only < 0 ? plane / (2 * g.num_kv_heads) : plane / g.num_kv_heads;
+    const int kv = kv_only < 0 ? (plane / g.num_kv_heads) & 1 : kv_only;
     const int tile_rows = kCompactThreads * kUnroll / g.row_vecs;      // >= 1, checked by the host
     cudaGridDependencySynchronize();        // the index list and the cache come from earlier work on the stream
     // One list for all layers (strides 0), or every layer of the range its own list and count.
     const int32_t* list = kPerLayer ? kept_pos + li * kept_stride : kept_pos;
     const int64_t n_all = __ldg(n_kept_ptr + (kPerLayer ? li * count_stride : 0));
-    if (blockIdx.x == 0 && threadIdx.x == 0 && kv == 0 && h == 0 && (kPerLayer || li == 0) && n_all > capacity)
+    if (blockIdx.x == 0 && threadIdx.x == 0 && (kv == 0 || kv_only > 0) && h == 0 && (kPerLayer || li == 0) &&
+        n_all > capacity)
         report(status_word, SHARPV_ERR_CAPACITY);
     const int64_t n = min(n_all, capacity);
     const char* s = src + (g.layer_begin + li) * g.src_layer + kv * g.src_kv + h * g.src_head;
@@ -264,7 +268,8 @@ namespace sharpv {
 sharpv_status kv_compact_launch(const void* kv_src, const sharpv_kv_layout* src_layout, void* kv_dst,
                                 const sharpv_kv_layout* dst_layout, int32_t layer_begin, int32_t layer_end,
                                 const int32_t* kept_pos, const int32_t* n_kept_ptr, int64_t kept_stride,
-                                int64_t count_stride, int64_t capacity, int32_t* status_word, cudaStream_t stream) {
+                                int64_t count_stride, int64_t capacity, int32_t* status_word, cudaStream_t stream,
+                                int kv_only) {
     if (!layout_ok(src_layout) || !layout_ok(dst_layout)) {
         if (src_layout && dst_layout && (!copy_dtype_ok(src_layout->dtype) || !copy_dtype_ok(dst_layout->dtype)))
             return SHARPV_ERR_UNSUPPORTED;
@@ -275,8 +280,9 @@ sharpv_status kv_compact_launch(const void* kv_src, const sharpv_kv_layout* src_
         return SHARPV_ERR_INVALID_ARG;
     if (layer_begin < 0 || layer_end > src_layout->num_layers || layer_begin > layer_end || capacity < 0)
         return SHARPV_ERR_INVALID_ARG;
-    if (!kv_src || !kv_dst || !n_kept_ptr) return SHARPV_ERR_INVALID_ARG;
+    if (!kv_src || !kv_dst || !n_kept_ptr || kv_only < -1 || kv_only > 1) return SHARPV_ERR_INVALID_ARG;
     const bool in_place = kv_src == kv_dst;
+    if (in_place && kv_only >= 0) return SHARPV_ERR_INVALID_ARG;
     if (in_place && (src_layout->stride_layer != dst_layout->stride_layer ||
                      src_layout->stride_kv != dst_layout->stride_kv ||
                      src_layout->stride_head != dst_layout->stride_head ||
@@ -343,9 +349,10 @@ sharpv_status kv_compact_launch(const void* kv_src, const sharpv_kv_layout* src_
     int64_t row_tiles = ((capacity + tile_rows - 1) / tile_rows + kGatherTilesPerCta - 1) / kGatherTilesPerCta;
     const int64_t most = kGatherMaxCtas / planes > 1 ? kGatherMaxCtas / planes : 1;
     if (row_tiles > most) row_tiles = most;
-    if (launch_dependent(kern, dim3((unsigned)row_tiles, (unsigned)planes), dim3(kCompactThreads), 0, stream,
+    const int planes_here = kv_only < 0 ? planes : planes / 2;
+    if (launch_dependent(kern, dim3((unsigned)row_tiles, (unsigned)planes_here), dim3(kCompactThreads), 0, stream,
                          (const char*)kv_src, (char*)kv_dst, g, kept_pos, n_kept_ptr, kept_stride,
-                         count_stride, capacity, status_word) != cudaSuccess) {
+                         count_stride, capacity, kv_only, status_word) != cudaSuccess) {
         (void)cudaGetLastError();
         return SHARPV_ERR_CUDA;
     }

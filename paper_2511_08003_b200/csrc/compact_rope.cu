@@ -15,6 +15,7 @@
 //                            vectors inside the rotary part also fetch their partner vector and the row's
 //                            cos / sin entries (L2-resident, shared by all planes)
 #include "common.cuh"
+#include "compact.cuh"
 
 #include <cuda_bf16.h>
 
@@ -168,8 +169,10 @@ kv_compact_rope_kernel(const char* __restrict__ src, char* __restrict__ dst, Rop
     }
 }
 
-// Tiles in (row tile, plane) order: tile = row_tile * planes + plane.  A CTA's run of tiles stays on one
-// row tile for as long as possible, so the table rows of that tile are read from global memory once.
+// The key planes of the call, plane = layer * heads + head (the value planes are bit copies and go through
+// the plain compaction kernel).  Tiles in (row tile, plane) order: tile = row_tile * planes + plane.  A
+// CTA's run of tiles stays on one row tile for as long as possible, so the table rows of that tile are read
+// from global memory once.
 template <int DT>
 __global__ void __launch_bounds__(kRopeThreads)
 kv_compact_rope_paired_kernel(const char* __restrict__ src, char* __restrict__ dst, RopeGeom g, int planes,
@@ -193,7 +196,8 @@ kv_compact_rope_paired_kernel(const char* __restrict__ src, char* __restrict__ d
     // where the run stands is stepped from tile to tile, not divided out again
     int64_t rt = t0 / planes;
     int plane = (int)(t0 - rt * planes);
-    int li = plane / (2 * g.num_kv_heads), kv = (plane / g.num_kv_heads) & 1, h = plane % g.num_kv_heads;
+    int li = plane / g.num_kv_heads, h = plane % g.num_kv_heads;
+    constexpr int kv = 0;
     // what a thread handles in every tile: vector vv of row rr of the tile (rows do not straddle warps)
     int rr[kRopeUnroll], vv[kRopeUnroll];
 #pragma unroll
@@ -282,10 +286,10 @@ kv_compact_rope_paired_kernel(const char* __restrict__ src, char* __restrict__ d
         if (++plane == planes) {
             plane = 0;
             ++rt;
-            li = 0; kv = 0; h = 0;
+            li = 0; h = 0;
         } else if (++h == g.num_kv_heads) {
             h = 0;
-            if (++kv == 2) { kv = 0; ++li; }
+            ++li;
         }
     }
 }
@@ -384,13 +388,18 @@ extern "C" sharpv_status sharpv_kv_compact_rope(
             (void)cudaGetLastError();
             return SHARPV_ERR_CUDA;
         }
-        if (launch_dependent(kern, dim3(grid), dim3(kRopeThreads), tab_bytes, stream, (const char*)kv_src,
-                             (char*)kv_dst, g, planes, kept_pos, kept_seq_offsets + num_seqs, capacity,
+        // keys here, values (half of the bytes, no arithmetic) through the plain compaction kernel
+        const int key_planes = planes / 2;
+        const int64_t key_tiles = (capacity + tile_rows - 1) / tile_rows * key_planes;
+        const unsigned key_grid = (unsigned)(key_tiles < want ? key_tiles : want);
+        if (launch_dependent(kern, dim3(key_grid), dim3(kRopeThreads), tab_bytes, stream, (const char*)kv_src,
+                             (char*)kv_dst, g, key_planes, kept_pos, kept_seq_offsets + num_seqs, capacity,
                              (const float2*)table, status_word) != cudaSuccess) {
             (void)cudaGetLastError();
             return SHARPV_ERR_CUDA;
         }
-        return SHARPV_OK;
+        return kv_compact_launch(kv_src, src_layout, kv_dst, dst_layout, layer_begin, layer_end, kept_pos,
+                                 kept_seq_offsets + num_seqs, 0, 0, capacity, status_word, stream, 1);
     }
     auto kern = src_layout->dtype == SHARPV_F32 ? kv_compact_rope_kernel<SHARPV_F32>
                                                  : kv_compact_rope_kernel<SHARPV_BF16>;
