@@ -25,7 +25,7 @@ namespace sharpv {
 namespace {
 
 constexpr int kRopeThreads = 256;
-constexpr int kRopeUnroll = 2;
+constexpr int kRopeUnroll = 4;
 constexpr int kRopeCtasPerSm = 4;
 
 struct RopeGeom {
