@@ -249,6 +249,42 @@ def test_kv_compact_layouts_and_layer_range():
     np.testing.assert_array_equal(to_host(dst_tm)[:, :, :kept.size], wl.kv[:, :, :, kept].transpose(0, 1, 3, 2, 4))
 
 
+@pytest.mark.parametrize("dtype,Dh", [(torch.bfloat16, 96), (torch.float32, 40), (torch.bfloat16, 8), (torch.float32, 516)])
+def test_kv_compact_row_sizes_that_are_not_a_power_of_two(dtype, Dh):
+    """Rows of 12, 10, 1 and 129 16-byte vectors (a tile of the copy kernels then holds a number of rows that does
+    not divide its vectors evenly): out of place, in place and with a capacity below the kept count, bit for bit
+    against the oracle; several row tiles, a ragged last tile."""
+    rng = np.random.default_rng(1200 + Dh)
+    L, H, T = 3, 2, 1500
+    kv = torch.randn((L, 2, H, T, Dh), dtype=torch.float32, device="cuda",
+                     generator=torch.Generator(device="cuda").manual_seed(Dh)).to(dtype)
+    kept = np.sort(rng.choice(T, size=701, replace=False)).astype(np.int32)
+    kept[:30] = np.arange(30)
+    kept = np.unique(kept)
+    n = kept.size
+    kept_d = torch.from_numpy(kept).cuda()
+    kso = torch.tensor([0, 400, n], dtype=torch.int32, device="cuda")
+    host = to_host(kv)
+    dst = torch.zeros((L, 2, H, n + 3, Dh), dtype=dtype, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sv.sharpv_kv_compact(kv, dst, kept_d, kso, capacity=n + 3, status_word=status)
+    torch.cuda.synchronize()
+    out = to_host(dst)
+    want = orc.kv_compact(host, kept)[:, :, :, :n]
+    np.testing.assert_array_equal(out[:, :, :, :n], want)
+    assert not out[:, :, :, n:].any() and int(status.item()) == 0
+    small = torch.zeros((L, 2, H, 100, Dh), dtype=dtype, device="cuda")
+    sv.sharpv_kv_compact(kv, small, kept_d, kso, capacity=100, layer_begin=1, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == sv.Status.ERR_CAPACITY
+    np.testing.assert_array_equal(to_host(small)[1:], want[1:, :, :, :100])
+    assert not to_host(small)[0].any()
+    inplace = kv.clone()
+    sv.sharpv_kv_compact(inplace, inplace, kept_d, kso, capacity=T)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(to_host(inplace), orc.kv_compact_inplace(host.copy(), kept))
+
+
 def test_kv_compact_rejects_partial_overlap_accepts_neighbours():
     """Source and destination carved out of one allocation: caches that touch without sharing a byte are
     compacted, a destination that starts inside the source is refused before anything is launched."""
