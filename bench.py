@@ -221,7 +221,7 @@ class ClockSampler:
 
     def __init__(self, index, period_s=0.005, pci_bus_id=None):
         import threading
-        self.samples, self.reason_bits, self.max_mhz = [], 0, None
+        self.samples, self.mem_samples, self.reason_bits, self.max_mhz, self.mem_max_mhz = [], [], 0, None, None
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -235,6 +235,7 @@ class ClockSampler:
             if self._h is None:
                 self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
             self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+            self.mem_max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_MEM))
         except Exception:
             self._nvml = None
             return
@@ -247,6 +248,7 @@ class ClockSampler:
         while not self._stop.is_set():
             try:
                 self.samples.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.mem_samples.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_MEM)))
                 self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
             except Exception:
                 pass
@@ -261,6 +263,9 @@ class ClockSampler:
         if self.samples:
             out["sm_mhz"] = statistics.median(self.samples)
             out["samples"] = len(self.samples)
+        if self.mem_samples:
+            out["mem_mhz"] = statistics.median(self.mem_samples)
+            out["mem_max_mhz"] = self.mem_max_mhz
         out["reasons"] = sorted(n for n, bit in self.REASONS.items() if self.reason_bits & bit)
         return out
 
@@ -612,6 +617,16 @@ def run_sharpv(args):
                    "note": "calibration + compaction on the survivors of stage one; token_budget = visual "
                            "tokens left after both stages / visual tokens in"}
         del c_kv, c_dst
+    # stage one and stage two each as one graph launch (stage two = calibration + compaction back to back)
+    stage_times = None
+    if not args.stage:
+        def stage_two(i=0):
+            path.stage_calibrate(i)
+            path.stage_compact(i)
+        path.stages["stage_two"] = stage_two
+        two = path.time_stage("stage_two", replays=10)
+        stage_times = {"stage_one_ms": round(kernels["prune"]["median_ms"], 5),
+                       "stage_two_ms": round(two["median_ms"], 5), "stage_two_best_ms": round(two["best_ms"], 5)}
     clocks = sampler.stop() if sampler else None
 
     total_ms = max_over_ranks(total_ms, dev, world)
@@ -724,6 +739,7 @@ def run_sharpv(args):
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "note": "tokens and hidden state copied from pinned host memory every step, kept-index lists "
                         "read back; the K/V cache is device-resident model state"},
+        "stage_times": stage_times,
         "gpu_launches": sum(LAUNCHES_PER_STEP[k] for k in STEP_STAGES) * replays,
         "clocks": clocks, "wall_s": round(wall, 3),
     }
